@@ -1,0 +1,134 @@
+/*
+ * bebop.h -- C ABI of the speculative rejection-sampling verify step
+ * (MTP draft-then-verify rollouts; "Breaking Entropy Bounds: Accelerating RL
+ * Training via MTP with Rejection Sampling", Sec. 2.2 and App. G.1).
+ *
+ * Conventions shared by every entry point
+ *   - Every tensor pointer, `workspace` included, is a DEVICE pointer owned by
+ *     the caller; scalars are passed by value.  The library never allocates,
+ *     frees or synchronises: work is enqueued on `cuda_stream` (a cudaStream_t
+ *     passed as void*, NULL = the legacy default stream) and outputs are valid
+ *     once that stream reaches the end of the call.
+ *   - Logits are row-major with the vocabulary contiguous.  `ld_*` is the
+ *     distance between consecutive rows in ELEMENTS (>= V).  Row (b,k) of a
+ *     [B,R,V] tensor starts at element (b*R + k) * ld.  The base pointer and
+ *     ld * sizeof(element) must be multiples of 16 bytes.
+ *   - -inf logits are legal (masked vocabulary, probability 0).
+ *   - Errors that can be seen on the host (NULL required pointer, B/K/V out of
+ *     range, K > BEBOP_MAX_K, ld < V, misalignment, workspace too small,
+ *     temperature_all <= 0 with no per-row tensor, device not sm_100) return a
+ *     status BEFORE any launch and write nothing.
+ *   - Data-dependent anomalies never trap; they set bits in row_status[b] and
+ *     the row still yields a defined result (see BEBOP_ROW_*).  A row with any
+ *     of the FATAL bits yields accept_len = 0, out_tokens = -1, tv = 0.
+ *   - Calls sharing one workspace must not overlap on the GPU.
+ */
+#ifndef BEBOP_H_
+#define BEBOP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BEBOP_MAX_K 32   /* accept bits of one sequence fit one warp ballot */
+
+typedef enum {
+    BEBOP_OK = 0,
+    BEBOP_ERR_NULL = 1,
+    BEBOP_ERR_SHAPE = 2,
+    BEBOP_ERR_DTYPE = 3,
+    BEBOP_ERR_ALIGN = 4,
+    BEBOP_ERR_WORKSPACE = 5,
+    BEBOP_ERR_TEMPERATURE = 6,
+    BEBOP_ERR_ARCH = 7,
+    BEBOP_ERR_CUDA = 8
+} bebop_status_t;
+
+typedef enum { BEBOP_F32 = 0, BEBOP_BF16 = 1 } bebop_dtype_t;
+
+/* bits of row_status[b] */
+#define BEBOP_ROW_NONFINITE 1   /* NaN or +inf logit in a row the method reads (FATAL)   */
+#define BEBOP_ROW_EMPTY 2       /* a row whose logits are all -inf (FATAL)                */
+#define BEBOP_ROW_BAD_TOKEN 4   /* draft token id outside [0,V) (FATAL)                   */
+#define BEBOP_ROW_ZERO_RESID 8  /* residual mass 0 at a rejected position: drew from p    */
+#define BEBOP_ROW_BAD_TEMP 16   /* per-row temperature <= 0 or non-finite (FATAL)         */
+#define BEBOP_ROW_WAIT_EXPIRED 32 /* a bounded device-side wait gave up (result undefined) */
+#define BEBOP_ROW_FATAL (1 | 2 | 4 | 16)
+
+/* Bytes of device scratch the three entry points below need for this shape
+ * (pure host function; 0 on invalid arguments).  The same buffer serves all
+ * three.  Must be 256-byte aligned. */
+size_t bebop_workspace_bytes(int B, int K, int V, bebop_dtype_t dt);
+
+/*
+ * Chain rejection-sampling verification (App. G.1, Algorithm 3), with logits in
+ * place of cached probabilities and the uniforms supplied by the caller.
+ * For each sequence b with L = draft_len[b] drafts and temperature tau_b:
+ *   p_k = softmax(target[b,k,:]/tau_b), q_k = softmax(draft[b,k,:]/tau_b)   (Sec. 2.2)
+ *   accept x_k while u_accept[b,k] * q_k(x_k) < p_k(x_k); stop at the first reject
+ *   at a reject at position n: draw y from max(0, p_n - q_n)/Z by inverse CDF,
+ *     y = min{ v : sum_{v'<=v} r(v') >= u_final[b] * Z }
+ *   if all L accepted: draw the bonus token the same way from p_L (target row L)
+ *   tv[b,k] = sum_v max(0, p_k - q_k) = d_TV(p_k, q_k) = 1 - E[accept]   (Eq. reject_sample)
+ * Rows k >= L are never read; the bonus row is read only when all L are accepted.
+ * The draw is evaluated in double precision so that it agrees with an fp64
+ * evaluation of the definition except on near-ties.
+ *
+ * target_logits [B,K+1,V], draft_logits [B,K,V] : dtype dt
+ * draft_tokens  [B,K] int32; draft_len [B] int32 in 0..K, or NULL (= K)
+ * temperature   [B] fp32, or NULL -> temperature_all (> 0) for every row
+ * u_accept [B,K], u_final [B] : fp32 uniforms in the open interval (0,1)
+ * accept_len [B], out_tokens [B,K+1] (x_1..x_n, y, then -1) : int32 outputs
+ * tv, p_draft, q_draft [B,K] fp32 outputs, each may be NULL (0 beyond draft_len)
+ * row_status [B] int32 output, may be NULL
+ */
+bebop_status_t bebop_verify(
+    const void* target_logits, int64_t ld_target,
+    const void* draft_logits, int64_t ld_draft,
+    const int32_t* draft_tokens, const int32_t* draft_len,
+    const float* temperature, float temperature_all,
+    const float* u_accept, const float* u_final,
+    int B, int K, int V, bebop_dtype_t dt,
+    int32_t* accept_len, int32_t* out_tokens,
+    float* tv, float* p_draft, float* q_draft, int32_t* row_status,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Total-variation distance of N independent row pairs (Eq. reject_sample and
+ * the identity of Sec. 3.3; forward value of the TV loss, App. F Algorithm 1):
+ *   tv[n]    = sum_v max(0, p - q), clamped to [0,1]
+ *   s_aux[n] = sum_v q(v) * 1[q(v) <= p(v)]   (the scalar S of Eq. tv_grad), may be NULL
+ * with p = softmax(target[n,:]/tau_n), q = softmax(draft[n,:]/tau_n).
+ * target_logits, draft_logits [N,V]; temperature [N] or NULL; row_status [N] or NULL.
+ */
+bebop_status_t bebop_tv(
+    const void* target_logits, int64_t ld_target,
+    const void* draft_logits, int64_t ld_draft,
+    const float* temperature, float temperature_all,
+    int N, int V, bebop_dtype_t dt,
+    float* tv, float* s_aux, int32_t* row_status,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Greedy-draft mode (the deterministic limit of target-only sampling, Sec. 2.2):
+ * g_k = lowest index attaining max_v target[b,k,v]; accept x_k while x_k == g_k;
+ * emit g at the stop position (g_L when all L drafts match).  All L+1 target
+ * rows of a sequence are read; temperature plays no role.
+ */
+bebop_status_t bebop_greedy_verify(
+    const void* target_logits, int64_t ld_target,
+    const int32_t* draft_tokens, const int32_t* draft_len,
+    int B, int K, int V, bebop_dtype_t dt,
+    int32_t* accept_len, int32_t* out_tokens, int32_t* row_status,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Static, host-side, human-readable name of a status code. */
+const char* bebop_status_string(bebop_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BEBOP_H_ */

@@ -1,0 +1,44 @@
+// Internal interface between the C-ABI entry points and the kernel launchers.
+#pragma once
+#include <climits>
+#include <cmath>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bebop_common.cuh"
+#include "bebop_layout.h"
+
+namespace bebop {
+
+// Addressing of the logit rows of a batch.  Verify: t_seq_rows = K+1,
+// d_seq_rows = K.  TV of N row pairs: B = N, K = 1, both = 1.
+struct RowArgs {
+    const char* target;
+    const char* draft;
+    int64_t t_row_bytes, d_row_bytes;   // ld * sizeof(element)
+    int64_t t_seq_rows, d_seq_rows;
+    const int32_t* draft_len;           // [B] or nullptr (= K)
+    const float* temperature;           // [B] or nullptr (= temperature_all)
+    float temperature_all;
+    int B, K, V, dt, nvec, nsplit;
+};
+
+struct VerifyOut {
+    int32_t* accept_len;   // [B]
+    int32_t* out_tokens;   // [B, K+1]
+    float* tv;             // [B, K] or nullptr
+    float* p_draft;        // [B, K] or nullptr
+    float* q_draft;        // [B, K] or nullptr
+    int32_t* row_status;   // [B] or nullptr
+};
+
+cudaError_t general_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                           const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                           cudaStream_t stream);
+cudaError_t general_tv(const RowArgs& a, const Plan& p, float* tv, float* s_aux, int32_t* row_status,
+                       char* ws, cudaStream_t stream);
+cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                           int32_t* accept_len, int32_t* out_tokens, int32_t* row_status, char* ws,
+                           cudaStream_t stream);
+
+}  // namespace bebop

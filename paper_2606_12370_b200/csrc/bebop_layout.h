@@ -1,0 +1,56 @@
+// Workspace layout and launch-shape decisions shared by the host entry points
+// and the kernels.  Plain host/device code, no CUDA calls.
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+namespace bebop {
+
+struct Plan {
+    int B, K, V, dt;
+    int nvec;        // 16-byte vectors per row (last one possibly ragged)
+    int nsplit;      // CTAs per row in the fp32 sweeps
+    int nsplit_d;    // CTAs per sequence in the fp64 draw
+    // byte offsets into the workspace (all 256-byte aligned)
+    size_t off_stats;   // float2 [B][K][2][nsplit]      (m, S) partials, fp32 sweep
+    size_t off_zpart;   // float2 [B][K][nsplit]         (Z, S_aux) partials
+    size_t off_stop;    // int    [B]                    stop position n, or -1 (fatal)
+    size_t off_dstats;  // double2[B][2][nsplit_d]       (m, S) partials, fp64
+    size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
+    size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
+    size_t off_fused;   // per-sequence records of the fused kernel
+    size_t total;
+};
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static inline Plan make_plan(int B, int K, int V, int dt) {
+    Plan p;
+    p.B = B; p.K = K; p.V = V; p.dt = dt;
+    const int vec = dt == 0 ? 4 : 8;
+    p.nvec = (V + vec - 1) / vec;
+    // fp32 sweeps: aim at >= 4 CTAs per SM over 2*B*K rows, slices of >= 256 vectors
+    long rows = (long)B * (K > 0 ? 2 * K : 1);
+    long want = (4L * 148 + rows - 1) / rows;
+    int cap = p.nvec / 256; if (cap < 1) cap = 1;
+    p.nsplit = (int)(want < 1 ? 1 : want);
+    if (p.nsplit > 32) p.nsplit = 32;
+    if (p.nsplit > cap) p.nsplit = cap;
+    long wantd = (8L * 148 + B - 1) / B;
+    p.nsplit_d = (int)(wantd < 1 ? 1 : wantd);
+    if (p.nsplit_d > 32) p.nsplit_d = 32;
+    if (p.nsplit_d > cap) p.nsplit_d = cap;
+    size_t o = 0;
+    const size_t Kk = (size_t)(K > 0 ? K : 1);
+    p.off_stats = o;  o = align256(o + sizeof(float) * 2 * (size_t)B * Kk * 2 * p.nsplit);
+    p.off_zpart = o;  o = align256(o + sizeof(float) * 2 * (size_t)B * Kk * p.nsplit);
+    p.off_stop = o;   o = align256(o + sizeof(int) * (size_t)B);
+    p.off_dstats = o; o = align256(o + sizeof(double) * 2 * (size_t)B * 2 * p.nsplit_d);
+    p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * p.nsplit_d);
+    p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
+    p.off_fused = o;  o = align256(o + 64 * (size_t)B);
+    p.total = o;
+    return p;
+}
+
+}  // namespace bebop
