@@ -168,8 +168,8 @@ __global__ void __launch_bounds__(kThreads) k_row_tv(RowArgs a, const float2* __
                 load_vec<DT>(qrow, iv, a.V, fq);
 #pragma unroll
                 for (int j = 0; j < VEC; ++j) {
-                    float p = ex2f((fp[j] - P.m) * c) * ip;
-                    float q = ex2f((fq[j] - Q.m) * c) * iq;
+                    float p = __fmul_rn(ex2f((fp[j] - P.m) * c), ip);
+                    float q = __fmul_rn(ex2f((fq[j] - Q.m) * c), iq);
                     float d = fmaxf(p - q, 0.f);
                     float sq = (q <= p) ? q : 0.f;
                     if (j & 1) { z1 += d; s1 += sq; } else { z0 += d; s0 += sq; }
@@ -263,9 +263,10 @@ __device__ __forceinline__ void draw_vec(const DrawRow& d, int iv, int V, double
     if (d.resid) load_vec<DT>(d.qrow, iv, V, fq);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-        double p = exp((double)fp[j] * d.inv_tau - d.mp) * d.ip;
+        // explicit roundings: a contracted p*ip - q would leave rounding dust when p == q
+        double p = __dmul_rn(exp((double)fp[j] * d.inv_tau - d.mp), d.ip);
         if (d.resid) {
-            double q = exp((double)fq[j] * d.inv_tau - d.mq) * d.iq;
+            double q = __dmul_rn(exp((double)fq[j] * d.inv_tau - d.mq), d.iq);
             double df = p - q;
             r[j] = df > 0.0 ? df : 0.0;
         } else {

@@ -15,15 +15,21 @@ def to_np(t):
     return None if t is None else t.detach().cpu().numpy()
 
 
-def oracle_on(x, idx=None, nthreads=0):
-    """Run the fp64 oracle on sequences `idx` (all when None) of a generated input set."""
-    sel = slice(None) if idx is None else torch.as_tensor(idx, device=x["target"].device)
-    tgt = x["target"][sel].float().cpu().numpy()
-    drf = x["draft"][sel].float().cpu().numpy()
-    pick = lambda t: None if t is None else to_np(t[sel])
-    return oracle.verify(tgt, drf, pick(x["draft_tokens"]), pick(x["u_accept"]), pick(x["u_final"]),
-                         draft_len=pick(x["draft_len"]), temperature=pick(x["temperature"]),
-                         temperature_all=x["temperature_all"], nthreads=nthreads)
+def oracle_on(x, idx=None, nthreads=0, chunk=32):
+    """Run the fp64 oracle on sequences `idx` (all when None) of a generated input set,
+    `chunk` sequences at a time so that the widened host copies stay small."""
+    B = x["target"].shape[0]
+    idx = np.arange(B) if idx is None else np.asarray(idx)
+    parts = []
+    for i0 in range(0, len(idx), chunk):
+        sel = torch.as_tensor(idx[i0:i0 + chunk], device=x["target"].device)
+        tgt = x["target"][sel].float().cpu().numpy()
+        drf = x["draft"][sel].float().cpu().numpy()
+        pick = lambda t: None if t is None else to_np(t[sel])
+        parts.append(oracle.verify(tgt, drf, pick(x["draft_tokens"]), pick(x["u_accept"]), pick(x["u_final"]),
+                                   draft_len=pick(x["draft_len"]), temperature=pick(x["temperature"]),
+                                   temperature_all=x["temperature_all"], nthreads=nthreads))
+    return {k: np.concatenate([p[k] for p in parts]) for k in parts[0]}
 
 
 def compare_verify(got, ref, dtype, idx=None, context=""):

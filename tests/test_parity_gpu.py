@@ -1,6 +1,7 @@
 """GPU parity: the CUDA path (through the C ABI) against the fp64 oracle on the
-same seeded tensors.  Small cases are compared sequence by sequence; full-size
-configurations on a sample of sequences plus size-independent invariants."""
+same seeded tensors, sequence by sequence.  Full-size configurations are compared
+on every sequence when the host has at least 8 cores (the oracle then needs a few
+seconds), otherwise on an evenly spaced sample plus size-independent invariants."""
 import numpy as np
 import pytest
 import torch
@@ -26,7 +27,7 @@ def full_check(cfg, pad_ld=0, draft_mode="sample", sample=None):
     torch.cuda.synchronize()
     check_properties(got, x)
     idx = None
-    if sample is not None and sample < cfg.B:
+    if sample is not None and sample < cfg.B and oracle.num_threads() < 8:
         idx = np.unique(np.linspace(0, cfg.B - 1, sample).astype(np.int64))
     ref = oracle_on(x, idx)
     return compare_verify(got, ref, cfg.dtype, idx, context=cfg.name), x, got
