@@ -59,8 +59,10 @@ typedef enum { BEBOP_F32 = 0, BEBOP_BF16 = 1 } bebop_dtype_t;
 #define BEBOP_ROW_FATAL (1 | 2 | 4 | 16)
 
 /* Bytes of device scratch the three entry points below need for this shape
- * (pure host function; 0 on invalid arguments).  The same buffer serves all
- * three.  Must be 256-byte aligned. */
+ * (pure host function; 0 on invalid arguments).  bebop_verify and
+ * bebop_greedy_verify of shape (B,K,V) use bebop_workspace_bytes(B,K,V,dt);
+ * bebop_tv of N rows uses bebop_workspace_bytes(N,1,V,dt).  The buffer must be
+ * 256-byte aligned; its contents need not be initialised. */
 size_t bebop_workspace_bytes(int B, int K, int V, bebop_dtype_t dt);
 
 /*
@@ -124,6 +126,17 @@ bebop_status_t bebop_greedy_verify(
     int B, int K, int V, bebop_dtype_t dt,
     int32_t* accept_len, int32_t* out_tokens, int32_t* row_status,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Test and measurement hooks (no counterpart in the paper).
+ * bebop_debug_force_general_path(1) makes bebop_verify use the split-row general
+ * kernels even for shapes the fused cluster kernel takes (process-wide switch).
+ * bebop_debug_fallback_offset returns the byte offset, inside the workspace of
+ * this shape, of an int32 that after a bebop_verify call through the fused kernel
+ * holds the number of sequences whose draw was re-done by the fp64 kernels.
+ */
+void bebop_debug_force_general_path(int on);
+size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
 
 /* Static, host-side, human-readable name of a status code. */
 const char* bebop_status_string(bebop_status_t status);

@@ -45,6 +45,10 @@ def load_library():
     lib.bebop_tv.argtypes = [vp, i64, vp, i64, vp, f32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     lib.bebop_greedy_verify.restype = i32
     lib.bebop_greedy_verify.argtypes = [vp, i64, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    lib.bebop_debug_force_general_path.restype = None
+    lib.bebop_debug_force_general_path.argtypes = [i32]
+    lib.bebop_debug_fallback_offset.restype = sz
+    lib.bebop_debug_fallback_offset.argtypes = [i32, i32, i32, i32]
     lib.bebop_status_string.restype = C.c_char_p
     lib.bebop_status_string.argtypes = [i32]
     _lib = lib
@@ -83,6 +87,14 @@ def _rows(t: torch.Tensor, ndim: int):
     return C.c_void_p(t.data_ptr()), int(ld)
 
 
+def bebop_debug_force_general_path(on: bool) -> None:
+    load_library().bebop_debug_force_general_path(1 if on else 0)
+
+
+def bebop_debug_fallback_offset(B: int, K: int, V: int, dt: int) -> int:
+    return int(load_library().bebop_debug_fallback_offset(B, K, V, dt))
+
+
 def bebop_workspace_bytes(B: int, K: int, V: int, dt: int) -> int:
     return int(load_library().bebop_workspace_bytes(B, K, V, dt))
 
@@ -90,7 +102,7 @@ def bebop_workspace_bytes(B: int, K: int, V: int, dt: int) -> int:
 def _workspace(B, K, V, dt, device, workspace):
     need = bebop_workspace_bytes(B, K, V, dt)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+        workspace = torch.zeros(max(need, 256), dtype=torch.uint8, device=device)
     return workspace, workspace.numel() * workspace.element_size()
 
 
@@ -135,6 +147,7 @@ def bebop_verify(target_logits, draft_logits, draft_tokens, u_accept, u_final, d
                             _ptr(res["accept_len"]), _ptr(res["out_tokens"]), _ptr(res["tv"]),
                             _ptr(res["p_draft"]), _ptr(res["q_draft"]), _ptr(res["row_status"]),
                             _ptr(ws), wsb, _stream()))
+    res["workspace"] = ws
     return res
 
 

@@ -7,6 +7,10 @@ using namespace bebop;
 
 namespace {
 
+// Test hook: route bebop_verify through the general (split-row) path even where the fused
+// kernel applies, so that both paths are covered by the parity tests.
+bool g_force_general = false;
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Compute capability of the current device, cached per device ordinal.
@@ -86,8 +90,13 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     RowArgs a = row_args(target_logits, ld_target, draft_logits, ld_draft, K + 1, K, draft_len,
                          temperature, temperature_all, B, K, V, dt, p);
     VerifyOut o{accept_len, out_tokens, tv, p_draft, q_draft, row_status};
-    cudaError_t e = general_verify(a, p, draft_tokens, u_accept, u_final, o,
-                                   static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSuccess;
+    bool launched = false;
+    if (!g_force_general && fused_supported(a))
+        e = fused_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
+    if (e == cudaSuccess && !launched) e = general_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
 
@@ -130,6 +139,13 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
     cudaError_t e = general_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status,
                                    static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
+}
+
+void bebop_debug_force_general_path(int on) { g_force_general = on != 0; }
+
+size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
+    if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;
+    return make_plan(B, K, V, (int)dt).off_fb;
 }
 
 const char* bebop_status_string(bebop_status_t status) {

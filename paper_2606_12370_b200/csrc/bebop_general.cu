@@ -10,6 +10,7 @@ namespace bebop {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kListSlots = 32;   // sequences in flight per pass of the list-driven draw
 constexpr float kNegInf = -INFINITY;
 
 __device__ __forceinline__ float tau_of(const RowArgs& a, int b) {
@@ -195,12 +196,16 @@ __global__ void __launch_bounds__(128) k_accept(RowArgs a, const float2* __restr
     if (b >= a.B) return;
     const int K = a.K, L = len_of(a, b);
     float tau = tau_of(a, b);
-    int st = tau_ok(tau) ? 0 : ST_BAD_TEMP;
     const bool active = lane < L;
     int tok = active ? draft_tokens[(int64_t)b * K + lane] : 0;
-    if (active && (tok < 0 || tok >= a.V)) st |= ST_BAD_TOKEN;
+    // precedence of the fatal conditions: bad temperature, then bad token id, then the
+    // first position whose rows are non-finite or empty
+    int st = 0;
+    if (!tau_ok(tau)) st = ST_BAD_TEMP;
+    else if (__ballot_sync(0xffffffffu, active && (tok < 0 || tok >= a.V))) st = ST_BAD_TOKEN;
     MS P{0.f, 1.f}, Q{0.f, 1.f};
     float z = 0.f;
+    int row_st = 0;
     if (active && st == 0) {
         const float c = kLog2e / tau;
         const float2* sp = stats + (((int64_t)b * K + lane) * 2) * a.nsplit;
@@ -212,10 +217,12 @@ __global__ void __launch_bounds__(128) k_accept(RowArgs a, const float2* __restr
             Q = ms_merge(Q, MS{w.x, w.y}, c);
             z += zp[s].x;
         }
-        st |= ms_status(P) | ms_status(Q);
+        row_st = ms_status(P) | ms_status(Q);
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) st |= __shfl_xor_sync(0xffffffffu, st, off);
+    {
+        unsigned badrows = __ballot_sync(0xffffffffu, row_st != 0);
+        if (badrows) st |= __shfl_sync(0xffffffffu, row_st, __ffs(badrows) - 1);
+    }
     if (st & ST_FATAL) {
         if (lane < K) {
             if (o.tv) o.tv[(int64_t)b * K + lane] = 0.f;
@@ -289,11 +296,10 @@ __device__ __forceinline__ bool draw_setup(const RowArgs& a, const int* stop, in
 
 // (m, S) in double of one slice of the stop row(s): S = sum exp(z/tau - m).
 template <int DT>
-__global__ void __launch_bounds__(kThreads) k_draw_stats(RowArgs a, const int* __restrict__ stop,
-                                                         int nsplit_d, double2* __restrict__ dstats) {
+__device__ __forceinline__ void draw_stats_body(const RowArgs& a, const int* __restrict__ stop, int b,
+                                                int split, int nsplit_d, double2* __restrict__ dstats,
+                                                double* shm, double* shs) {
     constexpr int VEC = Elem<DT>::VEC;
-    __shared__ double shm[kThreads / 32], shs[kThreads / 32];
-    int split = blockIdx.x % nsplit_d, b = blockIdx.x / nsplit_d;
     int n; bool resid; const char *prow, *qrow;
     if (!draw_setup(a, stop, b, &n, &resid, &prow, &qrow)) return;
     const double inv_tau = 1.0 / (double)tau_of(a, b);
@@ -337,6 +343,24 @@ __global__ void __launch_bounds__(kThreads) k_draw_stats(RowArgs a, const int* _
     }
 }
 
+// Sequences to draw for: all B, or the entries of a device-side list.
+struct DrawList {
+    const int* list;    // nullptr: every sequence 0..B-1
+    const int* count;   // number of list entries (device memory)
+};
+__device__ __forceinline__ int draw_items(const DrawList& dl, int B) { return dl.list ? min(*dl.count, B) : B; }
+__device__ __forceinline__ int draw_seq(const DrawList& dl, int i) { return dl.list ? dl.list[i] : i; }
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_draw_stats(RowArgs a, const int* __restrict__ stop,
+                                                         int nsplit_d, double2* __restrict__ dstats,
+                                                         DrawList dl) {
+    __shared__ double shm[kThreads / 32], shs[kThreads / 32];
+    const int split = blockIdx.x % nsplit_d, items = draw_items(dl, a.B);
+    for (int i = blockIdx.x / nsplit_d; i < items; i += gridDim.x / nsplit_d)
+        draw_stats_body<DT>(a, stop, draw_seq(dl, i), split, nsplit_d, dstats, shm, shs);
+}
+
 // Merge the fp64 partials of the stop row(s); returns status bits.
 __device__ __forceinline__ int draw_merge(const double2* dstats, int b, int nsplit_d, bool resid,
                                           DrawRow* d) {
@@ -371,11 +395,9 @@ __device__ __forceinline__ double slice_mass(const DrawRow& d, int V, int begin,
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads) k_draw_mass(RowArgs a, const int* __restrict__ stop,
-                                                        int nsplit_d, const double2* __restrict__ dstats,
-                                                        double* __restrict__ dmass) {
-    __shared__ double sh[kThreads / 32];
-    int split = blockIdx.x % nsplit_d, b = blockIdx.x / nsplit_d;
+__device__ __forceinline__ void draw_mass_body(const RowArgs& a, const int* __restrict__ stop, int b,
+                                               int split, int nsplit_d, const double2* __restrict__ dstats,
+                                               double* __restrict__ dmass, double* sh) {
     int n; DrawRow d;
     if (!draw_setup(a, stop, b, &n, &d.resid, &d.prow, &d.qrow)) return;
     d.inv_tau = 1.0 / (double)tau_of(a, b);
@@ -388,20 +410,36 @@ __global__ void __launch_bounds__(kThreads) k_draw_mass(RowArgs a, const int* __
     if (threadIdx.x == 0) *out = m;
 }
 
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_draw_mass(RowArgs a, const int* __restrict__ stop,
+                                                        int nsplit_d, const double2* __restrict__ dstats,
+                                                        double* __restrict__ dmass, DrawList dl) {
+    __shared__ double sh[kThreads / 32];
+    const int split = blockIdx.x % nsplit_d, items = draw_items(dl, a.B);
+    for (int i = blockIdx.x / nsplit_d; i < items; i += gridDim.x / nsplit_d)
+        draw_mass_body<DT>(a, stop, draw_seq(dl, i), split, nsplit_d, dstats, dmass, sh);
+}
+
 // Locate y = min{v : C(v) >= u * Z}: slice from the partials, thread chunk by a
 // scan of chunk sums, element by a sequential walk.  One block per sequence.
+struct PickShared {
+    double sh[kThreads / 32];
+    double part[32];
+    double cs[kThreads];
+    double t, c0;
+    int split, thread;
+};
+
 template <int DT>
-__global__ void __launch_bounds__(kThreads) k_draw_pick(RowArgs a, const int* __restrict__ stop,
-                                                        int nsplit_d, const double2* __restrict__ dstats,
-                                                        const double* __restrict__ dmass,
-                                                        const float* __restrict__ u_final, VerifyOut o) {
+__device__ __forceinline__ void draw_pick_body(const RowArgs& a, const int* __restrict__ stop, int b,
+                                               int nsplit_d, const double2* __restrict__ dstats,
+                                               const double* __restrict__ dmass,
+                                               const float* __restrict__ u_final, const VerifyOut& o,
+                                               PickShared& S) {
     constexpr int VEC = Elem<DT>::VEC;
-    __shared__ double sh[kThreads / 32];
-    __shared__ double part[32];
-    __shared__ double cs[kThreads];
-    __shared__ double sh_t, sh_c0;
-    __shared__ int sh_split, sh_thread;
-    const int b = blockIdx.x, K = a.K;
+    double* sh = S.sh; double* part = S.part; double* cs = S.cs;
+    double& sh_t = S.t; double& sh_c0 = S.c0; int& sh_split = S.split; int& sh_thread = S.thread;
+    const int K = a.K;
     int n; DrawRow d;
     if (!draw_setup(a, stop, b, &n, &d.resid, &d.prow, &d.qrow)) return;
     d.inv_tau = 1.0 / (double)tau_of(a, b);
@@ -500,6 +538,20 @@ __global__ void __launch_bounds__(kThreads) k_draw_pick(RowArgs a, const int* __
         }
         if (y < 0) y = lastpos;
         o.out_tokens[(int64_t)b * (K + 1) + n] = y;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_draw_pick(RowArgs a, const int* __restrict__ stop,
+                                                        int nsplit_d, const double2* __restrict__ dstats,
+                                                        const double* __restrict__ dmass,
+                                                        const float* __restrict__ u_final, VerifyOut o,
+                                                        DrawList dl) {
+    __shared__ PickShared S;
+    const int items = draw_items(dl, a.B);
+    for (int i = blockIdx.x; i < items; i += gridDim.x) {
+        draw_pick_body<DT>(a, stop, draw_seq(dl, i), nsplit_d, dstats, dmass, u_final, o, S);
+        __syncthreads();
     }
 }
 
@@ -652,9 +704,26 @@ cudaError_t general_verify(const RowArgs& a, const Plan& p, const int32_t* draft
         LAUNCH_DT(a.dt, k_row_tv, (unsigned)((int64_t)a.B * a.K * a.nsplit), kThreads, stream, a, stats, zpart);
     }
     k_accept<<<(a.B + 3) / 4, 128, 0, stream>>>(a, stats, zpart, o, draft_tokens, u_accept, stop, a.dt);
-    LAUNCH_DT(a.dt, k_draw_stats, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats);
-    LAUNCH_DT(a.dt, k_draw_mass, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats, dmass);
-    LAUNCH_DT(a.dt, k_draw_pick, (unsigned)a.B, kThreads, stream, a, stop, p.nsplit_d, dstats, dmass, u_final, o);
+    DrawList all{nullptr, nullptr};
+    LAUNCH_DT(a.dt, k_draw_stats, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats, all);
+    LAUNCH_DT(a.dt, k_draw_mass, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats, dmass, all);
+    LAUNCH_DT(a.dt, k_draw_pick, (unsigned)a.B, kThreads, stream, a, stop, p.nsplit_d, dstats, dmass, u_final, o, all);
+    return cudaGetLastError();
+}
+
+// fp64 draw for the sequences a device-side list names (the fused kernel's uncertain draws).
+// stop[b] holds the stop position of every listed sequence.  The split count is fixed at
+// kListSplit so that a handful of sequences still spreads over the whole GPU.
+cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
+                              const int* list, const int* count, cudaStream_t stream) {
+    int* stop = reinterpret_cast<int*>(ws + p.off_stop);
+    double2* dstats = reinterpret_cast<double2*>(ws + p.off_dstats);
+    double* dmass = reinterpret_cast<double*>(ws + p.off_dmass);
+    DrawList dl{list, count};
+    const int slots = a.B < kListSlots ? a.B : kListSlots;
+    LAUNCH_DT(a.dt, k_draw_stats, (unsigned)(slots * p.nsplit_l), kThreads, stream, a, stop, p.nsplit_l, dstats, dl);
+    LAUNCH_DT(a.dt, k_draw_mass, (unsigned)(slots * p.nsplit_l), kThreads, stream, a, stop, p.nsplit_l, dstats, dmass, dl);
+    LAUNCH_DT(a.dt, k_draw_pick, (unsigned)slots, kThreads, stream, a, stop, p.nsplit_l, dstats, dmass, u_final, o, dl);
     return cudaGetLastError();
 }
 

@@ -41,4 +41,14 @@ cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft
                            int32_t* accept_len, int32_t* out_tokens, int32_t* row_status, char* ws,
                            cudaStream_t stream);
 
+cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
+                              const int* list, const int* count, cudaStream_t stream);
+
+// Fused single-read cluster kernel (bebop_fused.cu).  fused_verify sets *launched = false and
+// does nothing when the shape or the device cannot take it; the caller then uses general_verify.
+bool fused_supported(const RowArgs& a);
+cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                         cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

@@ -11,6 +11,7 @@ struct Plan {
     int nvec;        // 16-byte vectors per row (last one possibly ragged)
     int nsplit;      // CTAs per row in the fp32 sweeps
     int nsplit_d;    // CTAs per sequence in the fp64 draw
+    int nsplit_l;    // CTAs per sequence in the list-driven fp64 draw (few sequences)
     // byte offsets into the workspace (all 256-byte aligned)
     size_t off_stats;   // float2 [B][K][2][nsplit]      (m, S) partials, fp32 sweep
     size_t off_zpart;   // float2 [B][K][nsplit]         (Z, S_aux) partials
@@ -18,7 +19,7 @@ struct Plan {
     size_t off_dstats;  // double2[B][2][nsplit_d]       (m, S) partials, fp64
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
-    size_t off_fused;   // per-sequence records of the fused kernel
+    size_t off_fb;      // int [1 + B]: count and list of sequences whose draw goes to fp64
     size_t total;
 };
 
@@ -40,15 +41,17 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.nsplit_d = (int)(wantd < 1 ? 1 : wantd);
     if (p.nsplit_d > 32) p.nsplit_d = 32;
     if (p.nsplit_d > cap) p.nsplit_d = cap;
+    p.nsplit_l = 32 < cap ? 32 : cap;
+    const int nsd = p.nsplit_d > p.nsplit_l ? p.nsplit_d : p.nsplit_l;
     size_t o = 0;
     const size_t Kk = (size_t)(K > 0 ? K : 1);
     p.off_stats = o;  o = align256(o + sizeof(float) * 2 * (size_t)B * Kk * 2 * p.nsplit);
     p.off_zpart = o;  o = align256(o + sizeof(float) * 2 * (size_t)B * Kk * p.nsplit);
     p.off_stop = o;   o = align256(o + sizeof(int) * (size_t)B);
-    p.off_dstats = o; o = align256(o + sizeof(double) * 2 * (size_t)B * 2 * p.nsplit_d);
-    p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * p.nsplit_d);
+    p.off_dstats = o; o = align256(o + sizeof(double) * 2 * (size_t)B * 2 * nsd);
+    p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
-    p.off_fused = o;  o = align256(o + 64 * (size_t)B);
+    p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
     p.total = o;
     return p;
 }

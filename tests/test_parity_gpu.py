@@ -15,6 +15,15 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+@pytest.fixture(autouse=True, params=["fused", "general"])
+def kernel_path(request):
+    """Every test runs twice: through the fused cluster kernel where the shape admits it,
+    and through the general split-row kernels."""
+    P.bebop_debug_force_general_path(request.param == "general")
+    yield request.param
+    P.bebop_debug_force_general_path(False)
+
+
 def run_verify(x, **kw):
     return P.bebop_verify(x["target"], x["draft"], x["draft_tokens"], x["u_accept"], x["u_final"],
                           draft_len=x["draft_len"], temperature=x["temperature"],
@@ -181,7 +190,8 @@ def test_deterministic_and_stream_ordered():
         b = run_verify(x)
     s.synchronize()
     for k in a:
-        assert torch.equal(a[k], b[k]), k
+        if k != "workspace":
+            assert torch.equal(a[k], b[k]), k
 
 
 # ------------------------------------------------------------------- bebop_tv
