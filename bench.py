@@ -134,7 +134,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "positions/s", "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "headline: B=256 K=3 V=151936 bf16 logits, tau=1 (oracle sample)"},
+        "config": {"workload": "headline: B=%d K=3 V=151936 bf16 logits, tau=1 (oracle sample)"},
         "cpu_baseline": {"value": val, "unit": "positions/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "positions/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -162,7 +162,8 @@ def run_ours(args):
 
     # weak scaling: every rank verifies its own batch of the headline shape (seed offset by rank)
     cfg = G.get_config(WORKLOAD)
-    cfg = G.get_config(WORKLOAD, seed=cfg.seed + 1000 * rank)
+    over = {"B": args.batch} if args.batch else {}
+    cfg = G.get_config(WORKLOAD, seed=cfg.seed + 1000 * rank, **over)
     x = G.make_inputs(cfg, dev)
     B, K, V = cfg.B, cfg.K, cfg.V
     es = 2 if cfg.dtype == "bf16" else 4
@@ -202,10 +203,10 @@ def run_ours(args):
     t1 = time.perf_counter()
     ms = e0.elapsed_time(e1)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = int(os.environ.get("BEBOP_LAUNCHES_PER_CALL", "6"))
+    launches_per_call = int(os.environ.get("BEBOP_LAUNCHES_PER_CALL", "4"))
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
-    e2e_steps = max(1, min(steps, 10))
+    e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))
     host = {k: x[k].cpu().pin_memory() for k in ("target", "draft", "draft_tokens", "u_accept", "u_final")}
     dev_in = {k: torch.empty_like(x[k]) for k in host}
     host_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype).pin_memory() for k in ("accept_len", "out_tokens", "tv")}
@@ -220,14 +221,14 @@ def run_ours(args):
             host_out[k].copy_(out[k], non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
-    for _ in range(2):
+    for _ in range(2 if e2e_steps else 0):
         e2e_step()
     barrier()
     w0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_step()
     barrier()
-    e2e_s = (time.perf_counter() - w0) / e2e_steps
+    e2e_s = (time.perf_counter() - w0) / max(e2e_steps, 1) if e2e_steps else float("inf")
     h2d = sum(host[k].numel() * host[k].element_size() for k in host)
     d2h = sum(host_out[k].numel() * host_out[k].element_size() for k in host_out)
 
@@ -247,8 +248,8 @@ def run_ours(args):
             "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": "headline: B=256 K=3 V=151936 bf16 logits, tau=1, N(0,3^2)+8 Zipf peaks, "
-                                   "draft=target+N(0,1), per GPU",
+            "config": {"workload": "headline: B=%d K=3 V=151936 bf16 logits, tau=1, N(0,3^2)+8 Zipf peaks, "
+                                   "draft=target+N(0,1), per GPU" % B,
                        "global_batch": world * B, "positions_per_step": world * positions,
                        "l2": "inputs (%.0f MB per GPU) larger than the 126 MB L2; no flush" % (alg_bytes / 1e6),
                        "draw": "fp64 inverse CDF at the stop row", "parallelism": "dp%d" % world},
@@ -283,6 +284,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="profiling aid: sequences per GPU instead of the workload's 256 (not a bench line)")
+    ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -136,6 +136,7 @@ bebop_status_t bebop_greedy_verify(
  * holds the number of sequences whose draw was re-done by the fp64 kernels.
  */
 void bebop_debug_force_general_path(int on);
+int bebop_debug_fused_clusters(bebop_dtype_t dt);   /* co-resident clusters the fused kernel gets on this device */
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
 
 /* Static, host-side, human-readable name of a status code. */

@@ -143,6 +143,10 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
 
 void bebop_debug_force_general_path(int on) { g_force_general = on != 0; }
 
+void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); }
+
+int bebop_debug_fused_clusters(bebop_dtype_t dt) { return fused_max_clusters((int)dt); }
+
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
     if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;
     return make_plan(B, K, V, (int)dt).off_fb;

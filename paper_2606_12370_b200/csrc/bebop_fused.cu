@@ -24,6 +24,7 @@
 // the same way.  Waits on the copy barriers are bounded; an expired wait sets
 // BEBOP_ROW_WAIT_EXPIRED and the kernel carries on (results undefined, flagged).
 #include "bebop_kernels.h"
+#include "bebop_ptx.cuh"
 
 namespace bebop {
 
@@ -33,83 +34,14 @@ constexpr int FT = 512;          // threads per CTA
 constexpr int CS = 8;            // CTAs per cluster
 constexpr int NWARP = FT / 32;
 constexpr int E_EMPTY = INT_MIN / 2;   // exponent reference of a slice without finite logits
-constexpr uint32_t kWaitPolls = 1u << 22;
+#ifndef BEBOP_TMA_CHUNK
+#define BEBOP_TMA_CHUNK 4096
+#endif
+constexpr uint32_t kChunk = BEBOP_TMA_CHUNK;   // bytes per bulk copy (multiple of 16)
 constexpr double kEClamp = 268435456.0;   // |max logit / tau * log2 e| beyond 2^28 saturates
 
 // flags exchanged per CTA slice
 constexpr int F_BAD = 1;         // NaN or +inf seen
-
-// ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ uint32_t cluster_id() { uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r; }
-__device__ __forceinline__ uint32_t num_clusters() { uint32_t r; asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r)); return r; }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
-    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
-}
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint4 v) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" :: "r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait; returns false if it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitPolls; ++i) if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t r; asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b)); return r;
-}
-__device__ __forceinline__ int redux_max(int v) {
-    int r; asm volatile("redux.sync.max.s32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v)); return r;
-}
-// order-preserving float <-> int map (canonical NaN sorts above +inf)
-__device__ __forceinline__ int f2ord(float f) { int b = __float_as_int(f); return b ^ ((b >> 31) & 0x7fffffff); }
-__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
-
-__device__ __forceinline__ double shfl_xor_d(double v, int m) { return __shfl_xor_sync(0xffffffffu, v, m); }
-__device__ __forceinline__ double shfl_up_d(double v, int d) { return __shfl_up_sync(0xffffffffu, v, d); }
-
-// max over the elements of one 16-byte vector, NaN-propagating
-template <int DT> __device__ __forceinline__ float vec_max(const uint4& v);
-template <> __device__ __forceinline__ float vec_max<0>(const uint4& v) {
-    return max_nan(max_nan(__uint_as_float(v.x), __uint_as_float(v.y)),
-                   max_nan(__uint_as_float(v.z), __uint_as_float(v.w)));
-}
-template <> __device__ __forceinline__ float vec_max<1>(const uint4& v) {
-    uint32_t m = max_nan_bf16x2(max_nan_bf16x2(v.x, v.y), max_nan_bf16x2(v.z, v.w));
-    return max_nan(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
-}
-// set the lanes at or beyond `keep` to -inf
-template <int DT> __device__ __forceinline__ void mask_tail(uint4& v, int keep) {
-    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
-    if (DT == 0) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) if (j >= keep) w[j] = kNegInfBits;
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j >= keep) w[j >> 1] = (j & 1) ? ((w[j >> 1] & 0x0000ffffu) | 0xff800000u)
-                                               : ((w[j >> 1] & 0xffff0000u) | 0x0000ff80u);
-    }
-}
 
 // ----------------------------------------------------------------- shared state
 struct __align__(16) Slot {      // per (parity, source rank): softmax partials of one item
@@ -155,7 +87,13 @@ struct FusedArgs {
     int* fb_count;
     int* fb_list;
     int vs;                              // vectors per CTA slice
+    long long* trace;                    // BEBOP_TRACE builds only: clock stamps of cluster 0
 };
+#ifdef BEBOP_TRACE
+#define TRACE(id) do { if (a.trace && cid == 0 && rank == 0 && tid == 0 && item < 60) a.trace[item * 16 + (id)] = clock64(); } while (0)
+#else
+#define TRACE(id) do {} while (0)
+#endif
 
 __device__ __forceinline__ float tau_of(const RowArgs& a, int b) { return a.temperature ? a.temperature[b] : a.temperature_all; }
 __device__ __forceinline__ bool tau_ok(float t) { return t > 0.f && t < INFINITY; }
@@ -239,13 +177,20 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
     if (tid == 0) { bonus_count = 0; bonus_overflow = 0; }
 
     auto issue = [&](int st, const char* prow, const char* qrow) {
-        // thread 0 only: arm the barrier and start the copies of this CTA's slice
+        // warp 0 only: lane 0 arms the barrier, then the lanes start the copies of this CTA's
+        // slice in chunks of kChunk bytes (many small bulk copies keep more requests in flight
+        // than one large one)
         if (nv_cta <= 0) return;
-        uint32_t bar = smem_u32(&S.full[st]);
-        uint32_t dst = smem_u32(stage + (size_t)st * 2 * ROW_BYTES);
-        mbar_expect_tx(bar, qrow ? 2 * slice_bytes : slice_bytes);
-        bulk_g2s(dst, prow + slice_off, slice_bytes, bar);
-        if (qrow) bulk_g2s(dst + ROW_BYTES, qrow + slice_off, slice_bytes, bar);
+        const uint32_t bar = smem_u32(&S.full[st]);
+        const uint32_t dst = smem_u32(stage + (size_t)st * 2 * ROW_BYTES);
+        if (lane == 0) mbar_expect_tx(bar, qrow ? 2 * slice_bytes : slice_bytes);
+        __syncwarp();
+        const uint32_t nchunk = (slice_bytes + kChunk - 1) / kChunk;
+        for (uint32_t cidx = lane; cidx < (qrow ? 2 * nchunk : nchunk); cidx += 32) {
+            const uint32_t row = cidx >= nchunk ? 1u : 0u, cc = cidx - row * nchunk;
+            const uint32_t off = cc * kChunk, len = min(kChunk, slice_bytes - off);
+            bulk_g2s(dst + row * ROW_BYTES + off, (row ? qrow : prow) + slice_off + off, len, bar);
+        }
     };
     auto trow = [&](int b, int k) { return R.target + ((int64_t)b * R.t_seq_rows + k) * R.t_row_bytes; };
     auto drow = [&](int b, int k) { return R.draft + ((int64_t)b * R.d_seq_rows + k) * R.d_row_bytes; };
@@ -266,7 +211,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
     // prologue: fill both stages
     uint32_t use[2] = {0, 0};                            // completed uses per stage (parity tracking)
     for (int s = 0; s < 2; ++s) {
-        if (ld.b < B) { if (tid == 0) issue(s, trow(ld.b, ld.k), drow(ld.b, ld.k)); next_item(ld); }
+        if (ld.b < B) { if (warp == 0) issue(s, trow(ld.b, ld.k), drow(ld.b, ld.k)); next_item(ld); }
     }
 
     // per-sequence state, identical in every thread of the cluster
@@ -288,7 +233,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
             // phase 1 is over for this cluster: both stages are free; start streaming bonus rows
             phase = 2;
             __syncthreads();
-            if (tid == 0) {
+            if (warp == 0) {
                 fence_proxy_async();
                 for (int s = 0; s < 2 && s < bonus_count; ++s) {
                     int bb = bonus_list[s];
@@ -303,6 +248,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
         else break;
         const int st = item & 1;
         const bool have_rows = b >= 0;
+        TRACE(0);
 
         float tau = 1.f;
         if (have_rows) tau = tau_of(R, b);
@@ -341,6 +287,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
                 if (!ok) S.wait_failed = 1;
             }
             use[st]++;
+            TRACE(1);
             const unsigned char* sp_ = stage + (size_t)st * 2 * ROW_BYTES;
 #pragma unroll
             for (int j = 0; j < NV; ++j) {
@@ -361,7 +308,8 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
             int op = redux_max(f2ord(mp)), oq = redux_max(f2ord(mq));
             if (lane == 0) { atomicMax(&S.wmax[st][0], op); atomicMax(&S.wmax[st][1], oq); }
             __syncthreads();                             // also: every read of the stage is done
-            if (tid == 0) {
+            TRACE(2);
+            if (warp == 0) {
                 // refill this stage with the item two ahead
                 fence_proxy_async();
                 if (phase == 1) {
@@ -406,6 +354,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
 #pragma unroll
                 for (int i = 0; i < NE; ++i) eq[i] = 0.f;
             }
+            TRACE(3);
             // block sums in double
             double dp = (double)s_p, dq = (double)s_q;
 #pragma unroll
@@ -424,6 +373,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
         if (phase == 1) { if (have_rows) next_item(ld); } else if (have_rows) { bonus_ld++; }
         // NOTE: in phase 2 the first two bonus items are issued when phase 2 begins (below).
 
+        TRACE(4);
         // ------------------------------------------------ exchange through DSMEM
         if (tid < CS) {
             // thread `tid` delivers this CTA's partials to CTA `tid`
@@ -440,14 +390,15 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
         __syncwarp();
         cluster_arrive();
         cluster_wait();
+        TRACE(5);
 
         // ------------------------------------------------ merge (warp 0), accept test (thread 0)
         if (warp == 0) {
             Slot sl;
             if (lane < CS) sl = S.slot[st][lane]; else { sl.sp = sl.sq = 0.0; sl.ep = sl.eq = E_EMPTY; sl.zprev = 0.f; sl.flags = 0; }
             int Em_p = redux_max(sl.ep), Em_q = redux_max(sl.eq);
-            double tp = sl.ep > E_EMPTY ? scalbn(sl.sp, max(sl.ep - Em_p, -2000)) : 0.0;
-            double tq = sl.eq > E_EMPTY ? scalbn(sl.sq, max(sl.eq - Em_q, -2000)) : 0.0;
+            double tp = sl.ep > E_EMPTY ? sl.sp * pow2d(max(sl.ep - Em_p, -2000)) : 0.0;
+            double tq = sl.eq > E_EMPTY ? sl.sq * pow2d(max(sl.eq - Em_q, -2000)) : 0.0;
             float zp = sl.zprev;
             int fl = sl.flags;
 #pragma unroll
@@ -471,8 +422,8 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
                 // this CTA's scale factors: p = e * 2^(Ep - Em_p) / Sp
                 float ac = 0.f, bc = 0.f;
                 if (have_rows && !bad) {
-                    ac = Ep > E_EMPTY ? (float)(scalbn(1.0, max(Ep - Em_p, -2000)) / Sp) : 0.f;
-                    if (pair) bc = Eq > E_EMPTY ? (float)(scalbn(1.0, max(Eq - Em_q, -2000)) / Sq) : 0.f;
+                    ac = Ep > E_EMPTY ? (float)(pow2d(max(Ep - Em_p, -2000)) * __drcp_rn(Sp)) : 0.f;
+                    if (pair) bc = Eq > E_EMPTY ? (float)(pow2d(max(Eq - Em_q, -2000)) * __drcp_rn(Sq)) : 0.f;
                 }
                 S.a_c = ac; S.b_c = bc;
                 int stop_here = 0;
@@ -498,6 +449,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
             }
         }
         __syncthreads();
+        TRACE(6);
         const int bad = S.bad;
         const int stop_here = S.stop_here;
         const float a_c = S.a_c, b_c = S.b_c;
@@ -568,6 +520,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
             my_zprev = pair && have_rows ? z : 0.f;
         }
 
+        TRACE(7);
         // record what the next exchange has to flush
         if (have_rows && pair) { prev_b = b; prev_k = k; prev_fatal = (seq_st & ST_FATAL) ? 1 : 0; }
         else prev_b = -1;
@@ -694,6 +647,7 @@ __global__ void __launch_bounds__(FT, 1) k_fused(const FusedArgs a) {
             }
             bonus_pos++;
         }
+        TRACE(8);
         ++item;
     }
 
@@ -760,10 +714,15 @@ int max_clusters() {
 // per cluster.
 bool fused_supported(const RowArgs& a) {
     constexpr int NV = 5;
-    if (a.nvec > CS * FT * NV) return false;
+    if (((((a.nvec + CS - 1) / CS) + 7) & ~7) > FT * NV) return false;
     if (a.nvec < 4 * CS) return false;
     return true;
 }
+
+long long* g_trace = nullptr;
+void fused_set_trace(long long* p) { g_trace = p; }
+
+int fused_max_clusters(int dt) { return dt == 0 ? max_clusters<0, 5>() : max_clusters<1, 5>(); }
 
 cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                          const float* u_accept, const float* u_final, VerifyOut o, char* ws,
@@ -779,7 +738,8 @@ cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_t
     fa.stop = reinterpret_cast<int*>(ws + p.off_stop);
     fa.fb_count = reinterpret_cast<int*>(ws + p.off_fb);
     fa.fb_list = fa.fb_count + 16;
-    fa.vs = (a.nvec + CS - 1) / CS;
+    fa.vs = (((a.nvec + CS - 1) / CS) + 7) & ~7;   // slices start on 128-byte boundaries
+    fa.trace = g_trace;
     cudaError_t e = cudaMemsetAsync(fa.fb_count, 0, sizeof(int), stream);
     if (e != cudaSuccess) return e;
     e = a.dt == 0 ? launch_fused<0, NV>(fa, ncl, stream) : launch_fused<1, NV>(fa, ncl, stream);

@@ -47,6 +47,8 @@ cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_fi
 // Fused single-read cluster kernel (bebop_fused.cu).  fused_verify sets *launched = false and
 // does nothing when the shape or the device cannot take it; the caller then uses general_verify.
 bool fused_supported(const RowArgs& a);
+int fused_max_clusters(int dt);
+void fused_set_trace(long long* p);
 cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                          const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                          cudaStream_t stream, bool* launched);
