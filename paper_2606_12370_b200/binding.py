@@ -88,7 +88,7 @@ def _rows(t: torch.Tensor, ndim: int):
 
 
 def bebop_debug_force_general_path(on: bool) -> None:
-    load_library().bebop_debug_force_general_path(1 if on else 0)
+    load_library().bebop_debug_force_general_path(int(on))
 
 
 def bebop_debug_fallback_offset(B: int, K: int, V: int, dt: int) -> int:

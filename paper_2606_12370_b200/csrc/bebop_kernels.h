@@ -53,4 +53,12 @@ cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_t
                          const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                          cudaStream_t stream, bool* launched);
 
+// Streaming cluster kernel (bebop_stream.cu): same contract as fused_verify.
+bool stream_supported(const RowArgs& a);
+int stream_max_clusters(int dt);
+void stream_set_trace(long long* p);
+cudaError_t stream_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                          const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                          cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

@@ -9,7 +9,7 @@
 
 namespace bebop {
 
-constexpr uint32_t kWaitPolls = 1u << 22;   // bound of every spin on an mbarrier
+constexpr uint32_t kWaitPolls = 1u << 20;   // bound of every spin on an mbarrier
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
@@ -44,6 +44,30 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// arrive on an mbarrier of another CTA of the cluster (address from mapa), release at cluster scope
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait with cluster-scope acquire; returns false if it gave up.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitPolls; ++i) if (mbar_try_wait_cluster(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, uint32_t x, uint32_t y) {
+    asm volatile("st.shared::cluster.v2.b32 [%0], {%1,%2};" :: "r"(addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void st_cluster_b32(uint32_t addr, uint32_t x) {
+    asm volatile("st.shared::cluster.b32 [%0], %1;" :: "r"(addr), "r"(x) : "memory");
+}
+__device__ __forceinline__ uint32_t redux_add(uint32_t v) {
+    uint32_t r; asm volatile("redux.sync.add.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v)); return r;
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
     uint32_t r; asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b)); return r;
@@ -70,19 +94,26 @@ template <> __device__ __forceinline__ float vec_max<1>(const uint4& v) {
     uint32_t m = max_nan_bf16x2(max_nan_bf16x2(v.x, v.y), max_nan_bf16x2(v.z, v.w));
     return max_nan(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
 }
-// set the lanes at or beyond `keep` to -inf
+// set the lanes at or beyond `keep` to -inf (register-only: no address is taken)
 template <int DT> __device__ __forceinline__ void mask_tail(uint4& v, int keep) {
-    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
     if (DT == 0) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) if (j >= keep) w[j] = kNegInfBits;
+        if (keep <= 0) v.x = kNegInfBits;
+        if (keep <= 1) v.y = kNegInfBits;
+        if (keep <= 2) v.z = kNegInfBits;
+        if (keep <= 3) v.w = kNegInfBits;
     } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j >= keep) w[j >> 1] = (j & 1) ? ((w[j >> 1] & 0x0000ffffu) | 0xff800000u)
-                                               : ((w[j >> 1] & 0xffff0000u) | 0x0000ff80u);
+        const uint32_t lo = 0x0000ff80u, hi = 0xff800000u;
+        if (keep <= 0) v.x = (v.x & 0xffff0000u) | lo;
+        if (keep <= 1) v.x = (v.x & 0x0000ffffu) | hi;
+        if (keep <= 2) v.y = (v.y & 0xffff0000u) | lo;
+        if (keep <= 3) v.y = (v.y & 0x0000ffffu) | hi;
+        if (keep <= 4) v.z = (v.z & 0xffff0000u) | lo;
+        if (keep <= 5) v.z = (v.z & 0x0000ffffu) | hi;
+        if (keep <= 6) v.w = (v.w & 0xffff0000u) | lo;
+        if (keep <= 7) v.w = (v.w & 0x0000ffffu) | hi;
     }
 }
+
 
 
 }  // namespace bebop
