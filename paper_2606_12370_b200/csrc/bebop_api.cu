@@ -9,7 +9,7 @@ namespace {
 
 // Test hook: route bebop_verify through the general (split-row) path even where the fused
 // kernel applies, so that both paths are covered by the parity tests.
-int g_path = 0;   // 0: streaming kernel where it applies, 1: general kernels, 2: lockstep fused kernel
+int g_path = 0;   // 0: ring kernel where it applies, 1: general kernels, 2: lockstep fused kernel, 3: register streaming kernel
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -94,7 +94,9 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 0 && stream_supported(a))
+    if (g_path == 0 && ring_supported(a))
+        e = ring_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
+    else if (g_path == 3 && stream_supported(a))
         e = stream_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
     else if (g_path == 2 && fused_supported(a))
         e = fused_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
@@ -145,9 +147,9 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
 
 void bebop_debug_force_general_path(int on) { g_path = on; }
 
-void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); stream_set_trace(static_cast<long long*>(p)); }
+void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); stream_set_trace(static_cast<long long*>(p)); ring_set_trace(static_cast<long long*>(p)); }
 
-int bebop_debug_fused_clusters(bebop_dtype_t dt) { return stream_max_clusters((int)dt); }
+int bebop_debug_fused_clusters(bebop_dtype_t dt) { return ring_max_clusters((int)dt); }
 
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
     if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;

@@ -61,4 +61,12 @@ cudaError_t stream_verify(const RowArgs& a, const Plan& p, const int32_t* draft_
                           const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                           cudaStream_t stream, bool* launched);
 
+// Ring kernel (bebop_ring.cu): tensor-memory rings, same contract as fused_verify.
+bool ring_supported(const RowArgs& a);
+int ring_max_clusters(int dt);
+void ring_set_trace(long long* p);
+cudaError_t ring_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

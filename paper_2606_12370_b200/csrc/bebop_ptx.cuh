@@ -116,4 +116,41 @@ template <int DT> __device__ __forceinline__ void mask_tail(uint4& v, int keep) 
 
 
 
+// ----------------------------------------------------------------- tensor memory
+// One warp allocates / frees all 512 columns of the SM's tensor memory.
+__device__ __forceinline__ void tmem_alloc512(uint32_t smem_result_addr) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_result_addr), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc512(uint32_t taddr) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(taddr), "r"(512u) : "memory");
+}
+__device__ __forceinline__ void tmem_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Each lane stores / loads 8 consecutive 32-bit columns of its own tensor-memory lane.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const float* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// 2^k as a float for k in [-126, 127] (0 below): exact
+__device__ __forceinline__ float pow2f(int k) { return k < -126 ? 0.f : __int_as_float((127 + k) << 23); }
+
+// ceil(x) for |x| < 2^22 without the conversion pipe: returns the integer and, in *r, the same value as a float
+__device__ __forceinline__ int ceil_alu(float x, float* r) {
+    const float magic = 12582912.f;               // 1.5 * 2^23
+    float y = x + magic;                          // round to nearest integer
+    int i = __float_as_int(y) - 0x4B400000;
+    float f = y - magic;
+    if (f < x) { f += 1.f; i += 1; }
+    *r = f;
+    return i;
+}
+
 }  // namespace bebop

@@ -113,7 +113,13 @@ __device__ __forceinline__ int row_status(int flagbit, int E, double S) {
 }  // namespace
 
 #ifdef BEBOP_TRACE
-#define TRACE(id) do { if (a.trace && cid == 0 && rank == 0 && tid == 0 && r < 60) a.trace[r * 16 + (id)] = clock64(); } while (0)
+#ifndef BEBOP_TRACE_TID
+#define BEBOP_TRACE_TID 0
+#endif
+#ifndef BEBOP_TRACE_RANK
+#define BEBOP_TRACE_RANK 0
+#endif
+#define TRACE(id) do { if (a.trace && cid == 0 && rank == BEBOP_TRACE_RANK && tid == BEBOP_TRACE_TID && r < 60) a.trace[r * 16 + (id)] = clock64(); } while (0)
 #else
 #define TRACE(id) do {} while (0)
 #endif
@@ -314,6 +320,7 @@ __global__ void __launch_bounds__(NT, 1) k_stream(const StreamArgs a) {
         int Ep = E_EMPTY, Eq = E_EMPTY, flags = 0;
         {
             uint4 rp[NV], rq[NV];
+            TRACE(9);
             if (nv_cta > 0 && !mbar_wait(smem_u32(&S.full[st]), (uint32_t)(r >> 1) & 1u)) S.wait_failed = 1;
             TRACE(1);
             const unsigned char* sp_ = stage + (size_t)st * 2 * ROW_BYTES;
@@ -329,11 +336,13 @@ __global__ void __launch_bounds__(NT, 1) k_stream(const StreamArgs a) {
                     rp[i] = neg_inf_vec<DT>(); rq[i] = neg_inf_vec<DT>();
                 }
             }
+            TRACE(10);
             float mp = vec_max<DT>(rp[0]), mq = vec_max<DT>(rq[0]);
 #pragma unroll
             for (int i = 1; i < NV; ++i) { mp = max_nan(mp, vec_max<DT>(rp[i])); mq = max_nan(mq, vec_max<DT>(rq[i])); }
             mp = ord2f(redux_max(f2ord(mp)));
             mq = ord2f(redux_max(f2ord(mq)));
+            TRACE(11);
             // this warp has consumed the stage: the last warp to say so refills it
             {
                 int last = 0;
@@ -360,6 +369,7 @@ __global__ void __launch_bounds__(NT, 1) k_stream(const StreamArgs a) {
                 if (mq != mq || mq == INFINITY) flags |= 2;
                 else if (mq != -INFINITY) { double t = fmin(fmax((double)mq * c64, -kEClamp), kEClamp); double E = ceil(t); Eq = (int)E; fq_ = (float)(E - t); mqu = mq; }
             }
+            TRACE(12);
             float s_p = 0.f, s_q = 0.f;
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
@@ -386,6 +396,7 @@ __global__ void __launch_bounds__(NT, 1) k_stream(const StreamArgs a) {
             long long fs_q = warp_sum_fixed(__double2ll_rn((double)s_q * kFix));
             if (flags & 1) fs_p = 0;
             if (flags & 2) fs_q = 0;
+            TRACE(13);
             int last = 0;
             if (lane == 0) {
                 WPart w; w.sp = fs_p; w.sq = fs_q; w.ep = Ep; w.eq = Eq; w.flags = flags; w.pad = 0;
