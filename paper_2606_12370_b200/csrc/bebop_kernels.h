@@ -69,4 +69,10 @@ cudaError_t ring_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);
 
+// Tile kernel (bebop_tile.cu): small vocabulary tiles, one CTA per tile; same contract.
+bool tile_supported(const RowArgs& a);
+cudaError_t tile_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched);
+
 }  // namespace bebop
