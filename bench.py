@@ -159,6 +159,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     P.load_library()
+    P.bebop_debug_force_general_path(args.path)
 
     # weak scaling: every rank verifies its own batch of the headline shape (seed offset by rank)
     cfg = G.get_config(WORKLOAD)
@@ -287,6 +288,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: sequences per GPU instead of the workload's 256 (not a bench line)")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
+    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default, 1 general kernels)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -94,7 +94,9 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 0 && tile_supported(a))
+    if (g_path == 0 && wave_supported(a))
+        e = wave_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
+    else if (g_path == 5 && tile_supported(a))
         e = tile_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
     else if (g_path == 4 && ring_supported(a))
         e = ring_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);

@@ -75,4 +75,10 @@ cudaError_t tile_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);
 
+// Wave kernel (bebop_wave.cu): persistent, ticket-scheduled, phases decoupled; same contract.
+bool wave_supported(const RowArgs& a);
+cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

@@ -6,6 +6,16 @@
 
 namespace bebop {
 
+// Workspace and schedule parameters of the wave kernel.
+constexpr int kWaveSliceVecs = 2048;   // 16-byte vectors per row slice, at most
+struct WavePlan {
+    int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
+    int wave_seqs, nwaves; // sequences per wave, waves
+    int lag;               // waves of stats work scheduled between a phase and the phase it depends on
+    size_t off_p1done, off_adone, off_p2done, zero_bytes;
+    size_t off_part, off_rstat, off_zpart, off_dpart, off_sinfo, total;
+};
+
 struct Plan {
     int B, K, V, dt;
     int nvec;        // 16-byte vectors per row (last one possibly ragged)
@@ -21,6 +31,7 @@ struct Plan {
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
     size_t off_fb;      // int [1 + B]: count and list of sequences whose draw goes to fp64
     size_t off_tile;    // workspace of the tile kernel
+    size_t off_wave;    // workspace of the wave kernel
     size_t total;
 };
 
@@ -40,6 +51,33 @@ static inline size_t tile_ws_bytes(int B, int K, int nvec) {
     return tile_ws_zero_bytes(B, K) + align256(32 * rows * T) + align256(4 * rows * T) + align256(16 * (size_t)B * T);
 }
 
+static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
+    (void)dt;
+    WavePlan w;
+    w.T = (nvec + kWaveSliceVecs - 1) / kWaveSliceVecs; if (w.T < 1) w.T = 1;
+    w.slice_vecs = (((nvec + w.T - 1) / w.T) + 7) & ~7;
+    const size_t NR = (size_t)(2 * K + 1);
+    const size_t seq_bytes = NR * (size_t)nvec * 16;
+    size_t ws = ((size_t)18 << 20) / (seq_bytes ? seq_bytes : 1);
+    if (ws < 1) ws = 1;
+    if (ws > (size_t)B) ws = (size_t)B;
+    w.wave_seqs = (int)ws;
+    w.nwaves = (B + w.wave_seqs - 1) / w.wave_seqs;
+    w.lag = 2;
+    size_t o = 256;                                           // ticket, wait flag
+    w.off_p1done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
+    w.off_adone = o;  o += align256(sizeof(int) * (size_t)w.nwaves);
+    w.off_p2done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
+    w.zero_bytes = o;
+    w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
+    w.off_rstat = o;  o += align256(32 * (size_t)B * NR);
+    w.off_zpart = o;  o += align256(4 * (size_t)B * (K > 0 ? K : 1) * w.T);
+    w.off_dpart = o;  o += align256(16 * (size_t)B * w.T);
+    w.off_sinfo = o;  o += align256(16 * (size_t)B);
+    w.total = o;
+    return w;
+}
+
 static inline Plan make_plan(int B, int K, int V, int dt) {
     Plan p;
     p.B = B; p.K = K; p.V = V; p.dt = dt;
@@ -47,7 +85,7 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.nvec = (V + vec - 1) / vec;
     // fp32 sweeps: aim at >= 4 CTAs per SM over 2*B*K rows, slices of >= 256 vectors
     long rows = (long)B * (K > 0 ? 2 * K : 1);
-    long want = (4L * 148 + rows - 1) / rows;
+    long want = (4L * 148 * 8 + rows - 1) / rows;   // about four full waves of 8 CTAs per SM
     int cap = p.nvec / 256; if (cap < 1) cap = 1;
     p.nsplit = (int)(want < 1 ? 1 : want);
     if (p.nsplit > 32) p.nsplit = 32;
@@ -68,6 +106,7 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
     p.off_tile = o;   o = align256(o + tile_ws_bytes(B, K, p.nvec));
+    p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
     p.total = o;
     return p;
 }

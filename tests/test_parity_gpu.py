@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.fixture(autouse=True, params=["tile", "general"])
+@pytest.fixture(autouse=True, params=["wave", "general"])
 def kernel_path(request):
     """Every test runs twice: through the fused cluster kernel where the shape admits it,
     and through the general split-row kernels."""
