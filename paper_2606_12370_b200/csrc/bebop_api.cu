@@ -151,7 +151,7 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
 
 void bebop_debug_force_general_path(int on) { g_path = on; }
 
-void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); stream_set_trace(static_cast<long long*>(p)); ring_set_trace(static_cast<long long*>(p)); }
+void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); stream_set_trace(static_cast<long long*>(p)); ring_set_trace(static_cast<long long*>(p)); wave_set_trace(static_cast<long long*>(p)); }
 
 int bebop_debug_fused_clusters(bebop_dtype_t dt) { return ring_max_clusters((int)dt); }
 

@@ -77,6 +77,7 @@ cudaError_t tile_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
 
 // Wave kernel (bebop_wave.cu): persistent, ticket-scheduled, phases decoupled; same contract.
 bool wave_supported(const RowArgs& a);
+void wave_set_trace(long long* p);
 cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);

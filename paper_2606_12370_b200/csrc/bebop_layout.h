@@ -55,7 +55,7 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
     (void)dt;
     WavePlan w;
     w.T = (nvec + kWaveSliceVecs - 1) / kWaveSliceVecs; if (w.T < 1) w.T = 1;
-    w.slice_vecs = (((nvec + w.T - 1) / w.T) + 7) & ~7;
+    w.slice_vecs = (((nvec + w.T - 1) / w.T) + 15) & ~15;   // halves (phase P2) stay 128-byte aligned
     const size_t NR = (size_t)(2 * K + 1);
     const size_t seq_bytes = NR * (size_t)nvec * 16;
     size_t ws = ((size_t)18 << 20) / (seq_bytes ? seq_bytes : 1);
@@ -71,8 +71,8 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
     w.zero_bytes = o;
     w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
     w.off_rstat = o;  o += align256(32 * (size_t)B * NR);
-    w.off_zpart = o;  o += align256(4 * (size_t)B * (K > 0 ? K : 1) * w.T);
-    w.off_dpart = o;  o += align256(16 * (size_t)B * w.T);
+    w.off_zpart = o;  o += align256(4 * (size_t)B * (K > 0 ? K : 1) * 2 * w.T);
+    w.off_dpart = o;  o += align256(16 * (size_t)B * 2 * w.T);
     w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.total = o;
     return w;

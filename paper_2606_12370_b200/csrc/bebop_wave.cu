@@ -74,6 +74,7 @@ struct WaveArgs {
     DPart* dpart;         // [B][T]
     SeqInfo* sinfo;       // [B]
     int ntickets, lag;
+    long long* trace;
     int T, slice_vecs, wave_seqs, nwaves;
 };
 
@@ -140,7 +141,7 @@ __device__ __forceinline__ const char* row_ptr(const RowArgs& R, int b, int r) {
 // ------------------------------------------------------------------ phase P1
 template <int DT>
 __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b, int r, int s) {
-    constexpr int VEC = Elem<DT>::VEC, U = 4;
+    constexpr int VEC = Elem<DT>::VEC, NV = SLICE_VECS / WT;     // 8 vectors per thread
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = len_of(R, b), K = R.K;
@@ -153,44 +154,40 @@ __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b
     const int nv = max(min(a.slice_vecs, R.nvec - v0), 0);
     const char* row = row_ptr(R, b, r) + (int64_t)v0 * 16;
 
-    float m_ref = -INFINITY, frac = 0.f;
+    // every load of the task is issued before anything is used
+    uint4 raw[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        const int v = tid + u * WT;
+        raw[u] = neg_inf_vec<DT>();
+        if (v < nv) raw[u] = ldg16_stream(row + (size_t)v * 16);
+    }
+    if ((v0 + nv) * VEC > R.V) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int gbase = (v0 + tid + u * WT) * VEC;
+            if (tid + u * WT < nv && gbase + VEC > R.V) mask_tail<DT>(raw[u], R.V - gbase);
+        }
+    }
+    float m = vec_max<DT>(raw[0]);
+#pragma unroll
+    for (int u = 1; u < NV; ++u) m = max_nan(m, vec_max<DT>(raw[u]));
+    const bool bad = m != m || m == INFINITY;
     int E = E_EMPTY;
+    float frac = 0.f, m_ref = 0.f;
+    if (!bad && m != -INFINITY) { reference(m, c, &E, &frac); m_ref = m; }
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    bool bad = false;
-    for (int i0 = tid; i0 < nv; i0 += WT * U) {
-        uint4 raw[U];
+    if (E > E_EMPTY) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int v = i0 + u * WT;
-            raw[u] = neg_inf_vec<DT>();
-            if (v < nv) {
-                raw[u] = ldg16_stream(row + (size_t)v * 16);
-                const int gbase = (v0 + v) * VEC;
-                if (gbase + VEC > R.V) mask_tail<DT>(raw[u], R.V - gbase);
-            }
-        }
-        float bm = max_nan(max_nan(vec_max<DT>(raw[0]), vec_max<DT>(raw[1])), max_nan(vec_max<DT>(raw[2]), vec_max<DT>(raw[3])));
-        if (bm != bm || bm == INFINITY) bad = true;
-        else if (bm > m_ref) {
-            // new reference point: rescale the running sums by an exact power of two
-            int En; float fn;
-            reference(bm, c, &En, &fn);
-            const float sc = E > E_EMPTY ? pow2f(max(E - En, -126)) : 0.f;
-            s0 *= sc; s1 *= sc; s2 *= sc; s3 *= sc;
-            E = En; frac = fn; m_ref = bm;
-        }
-        if (E > E_EMPTY) {
+        for (int u = 0; u < NV; ++u) {
+            float f[VEC];
+            unpack<DT>(raw[u], f);
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                float f[VEC];
-                unpack<DT>(raw[u], f);
-#pragma unroll
-                for (int i = 0; i < VEC; i += 4) {
-                    s0 += ex2f(fmaf(f[i] - m_ref, c, -frac));
-                    s1 += ex2f(fmaf(f[i + 1] - m_ref, c, -frac));
-                    s2 += ex2f(fmaf(f[i + 2] - m_ref, c, -frac));
-                    s3 += ex2f(fmaf(f[i + 3] - m_ref, c, -frac));
-                }
+            for (int i = 0; i < VEC; i += 4) {
+                s0 += ex2f(fmaf(f[i] - m_ref, c, -frac));
+                s1 += ex2f(fmaf(f[i + 1] - m_ref, c, -frac));
+                s2 += ex2f(fmaf(f[i + 2] - m_ref, c, -frac));
+                s3 += ex2f(fmaf(f[i + 3] - m_ref, c, -frac));
             }
         }
     }
@@ -200,7 +197,7 @@ __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b
     st = E > E_EMPTY ? st * pow2f(max(E - Ew, -126)) : 0.f;
     st = warp_sum(st);
     const unsigned anybad = __ballot_sync(0xffffffffu, bad);
-    float mw = ord2f(redux_max(f2ord(m_ref)));
+    float mw = ord2f(redux_max(f2ord(bad ? -INFINITY : m)));
     if (anybad) mw = __int_as_float(0x7fc00000);
     if (lane == 0) { S.redf[0][warp] = st; S.redi[warp] = Ew; S.redf[1][warp] = mw; }
     __syncthreads();
@@ -260,61 +257,83 @@ __device__ __forceinline__ void phase_a(const WaveArgs& a, WaveShared& S, int b)
         }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (warp == 0) {
+        // lane k owns draft position k (K <= 32): tokens, gathered logits, accept bit; ballots give the chain
+        const bool active = lane < L;
+        const int tk = active ? a.draft_tokens[(int64_t)b * K + lane] : 0;
         int seq_st = ok ? 0 : ST_BAD_TEMP;
-        if (!seq_st)
-            for (int j = 0; j < L; ++j) { int tk = a.draft_tokens[(int64_t)b * K + j]; if (tk < 0 || tk >= V) seq_st = ST_BAD_TOKEN; }
-        int n = L, alive = 1;
-        for (int k = 0; k < L && !(seq_st & ST_FATAL); ++k) {
-            const int rs = sh_status[k] | sh_status[K + 1 + k];
-            if (rs) { seq_st |= rs; break; }              // the first bad row pair decides
-            const int tk = a.draft_tokens[(int64_t)b * K + k];
-            const float zpx = DT == 0 ? load_one<0>(row_ptr(R, b, k), tk) : load_one<1>(row_ptr(R, b, k), tk);
-            const float zqx = DT == 0 ? load_one<0>(row_ptr(R, b, K + 1 + k), tk) : load_one<1>(row_ptr(R, b, K + 1 + k), tk);
+        if (!seq_st && __ballot_sync(0xffffffffu, active && (tk < 0 || tk >= V))) seq_st = ST_BAD_TOKEN;
+        // the first bad row pair decides the status; rows after it do not count
+        const int rs = active ? (sh_status[lane] | sh_status[K + 1 + lane]) : 0;
+        const unsigned badrows = __ballot_sync(0xffffffffu, rs != 0);
+        const int first_bad = badrows ? __ffs(badrows) - 1 : 32;
+        if (!seq_st && badrows) seq_st = __shfl_sync(0xffffffffu, rs, first_bad);
+        double px = 0.0, qx = 0.0;
+        bool acc = false;
+        if (active && !(seq_st & ST_FATAL) && lane < first_bad) {
+            const float zpx = DT == 0 ? load_one<0>(row_ptr(R, b, lane), tk) : load_one<1>(row_ptr(R, b, lane), tk);
+            const float zqx = DT == 0 ? load_one<0>(row_ptr(R, b, K + 1 + lane), tk) : load_one<1>(row_ptr(R, b, K + 1 + lane), tk);
             const double cd = (double)c;
-            const double px = exp2((double)zpx * cd - (double)sh_E[k]) / sh_S[k];
-            const double qx = exp2((double)zqx * cd - (double)sh_E[K + 1 + k]) / sh_S[K + 1 + k];
-            if (a.o.p_draft) a.o.p_draft[(int64_t)b * K + k] = (float)px;
-            if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + k] = (float)qx;
-            if (alive && !((double)a.u_accept[(int64_t)b * K + k] * qx < px)) { alive = 0; n = k; }
+            px = exp2((double)zpx * cd - (double)sh_E[lane]) / sh_S[lane];
+            qx = exp2((double)zqx * cd - (double)sh_E[K + 1 + lane]) / sh_S[K + 1 + lane];
+            acc = (double)a.u_accept[(int64_t)b * K + lane] * qx < px;
         }
-        if (!(seq_st & ST_FATAL) && alive && sh_status[L]) seq_st |= sh_status[L];   // bonus row, read only now
+        const unsigned rej = __ballot_sync(0xffffffffu, active && !acc);
+        int n = rej ? __ffs(rej) - 1 : L;
+        if (!(seq_st & ST_FATAL) && n == L && sh_status[L]) seq_st |= sh_status[L];   // bonus row, read only now
         const bool fatal = (seq_st & ST_FATAL) != 0;
-        // integer outputs (position n is filled by the draw)
         const int nn = fatal ? 0 : n;
-        a.o.accept_len[b] = nn;
-        for (int q = 0; q <= K; ++q)
-            if (fatal || q != nn) a.o.out_tokens[(int64_t)b * (K + 1) + q] = q < nn ? a.draft_tokens[(int64_t)b * K + q] : -1;
-        if (a.o.row_status) a.o.row_status[b] = seq_st;
-        a.stop[b] = fatal ? -1 : nn;
-        for (int q = 0; q < K; ++q) {
-            if (fatal || q >= L) {
-                if (a.o.tv) a.o.tv[(int64_t)b * K + q] = 0.f;
-                if (a.o.p_draft) a.o.p_draft[(int64_t)b * K + q] = 0.f;
-                if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + q] = 0.f;
-            }
+        // outputs: lane q writes position q (position nn is filled by the draw)
+        for (int q = lane; q <= K; q += 32)
+            if (fatal || q != nn) a.o.out_tokens[(int64_t)b * (K + 1) + q] = q < nn ? tk : -1;   // q < nn <= 32: q == lane
+        if (lane < K) {
+            const bool zero = fatal || lane >= L;
+            if (a.o.p_draft) a.o.p_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)px;
+            if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)qx;
+            if (zero && a.o.tv) a.o.tv[(int64_t)b * K + lane] = 0.f;
         }
-        // normalisers for phase P2: 2^(x*c - E) is evaluated as 2^((x - m_ref)*c - frac) around the row maximum
-        float sys = 0.f;
-        for (int r = 0; r < NR; ++r) {
-            RowStat rs; rs.inv_s = 0.0; rs.m_ref = 0.f; rs.frac = 0.f; rs.e = sh_E[r]; rs.pad = 0;
+        // normalisers for phase P2: 2^(x*c - E) is evaluated as 2^((x - m_ref)*c - frac) around the row maximum;
+        // lane r (and r + 32, r + 64) owns row r
+        double my_inv[3] = {0.0, 0.0, 0.0};
+        for (int i = 0, r = lane; r < NR; r += 32, ++i) {
+            RowStat st; st.inv_s = 0.0; st.m_ref = 0.f; st.frac = 0.f; st.e = sh_E[r]; st.pad = 0;
             if (!fatal && sh_E[r] > E_EMPTY && sh_S[r] > 0.0) {
-                rs.inv_s = 1.0 / sh_S[r];
+                st.inv_s = 1.0 / sh_S[r];
                 int Er; float fr;
                 reference(sh_M[r], c, &Er, &fr);           // Er == sh_E[r]: the row maximum fixes the exponent
-                rs.m_ref = sh_M[r]; rs.frac = fr + (float)(sh_E[r] - Er);
+                st.m_ref = sh_M[r]; st.frac = fr + (float)(sh_E[r] - Er);
             }
-            a.rstat[(int64_t)b * NR + r] = rs;
+            a.rstat[(int64_t)b * NR + r] = st;
+            if (i < 3) my_inv[i] = st.inv_s;
         }
+        // |fl(1/S) - 1/S| / (1/S) of the rows the draw uses: what the fp32 scale factors add to a prefix sum
         const int draw_row = fatal ? -1 : nn;
+        float sys = 0.f;
         if (draw_row >= 0) {
-            // |fl(1/S) - 1/S| / (1/S), an upper bound of what the fp32 scale factors add to a prefix sum
-            const double ip = a.rstat[(int64_t)b * NR + draw_row].inv_s;
-            sys += (float)(fabs((double)(float)ip - ip) / ip);
-            if (draw_row < L) { const double iq = a.rstat[(int64_t)b * NR + K + 1 + draw_row].inv_s; sys += (float)(fabs((double)(float)iq - iq) / iq); }
+            const int rp_ = draw_row, rq_ = draw_row < L ? K + 1 + draw_row : -1;
+            double ip = 0.0, iq = 0.0;
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                const double v = my_inv[i];
+                const double vp = __shfl_sync(0xffffffffu, v, rp_ & 31);
+                const double vq = __shfl_sync(0xffffffffu, v, (rq_ < 0 ? 0 : rq_) & 31);
+                if ((rp_ >> 5) == i) ip = vp;
+                if (rq_ >= 0 && (rq_ >> 5) == i) iq = vq;
+            }
+            if (ip > 0.0) sys += (float)(fabs((double)(float)ip - ip) / ip);
+            if (iq > 0.0) sys += (float)(fabs((double)(float)iq - iq) / iq);
         }
-        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = draw_row; si.sys = sys; si.pad = 0;
-        a.sinfo[b] = si;
+        if (lane == 0) {
+            a.o.accept_len[b] = nn;
+            if (a.o.row_status) a.o.row_status[b] = seq_st;
+            a.stop[b] = fatal ? -1 : nn;
+            SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = draw_row; si.sys = sys; si.pad = 0;
+            a.sinfo[b] = si;
+        }
+        __syncwarp();
+        // everything phase P2 reads was written by this warp: lane 0's release (in the caller) must cover
+        // the other lanes' stores
+        __threadfence();
     }
 }
 
@@ -339,53 +358,54 @@ __device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, b
 }
 
 // ------------------------------------------------------------------ phase P2
+// Slices of phase P2 and D are half as long as those of P1 (two rows are in flight per thread).
 template <int DT>
 __device__ __forceinline__ void phase_p2(const WaveArgs& a, WaveShared& S, int b, int k, int s) {
-    constexpr int VEC = Elem<DT>::VEC;
+    constexpr int VEC = Elem<DT>::VEC, NV = SLICE_VECS / (2 * WT);    // 4 vectors per thread and row
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1;
+    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1, T2 = 2 * a.T, sv = a.slice_vecs >> 1;
     if (k > L) return;
     const SeqInfo si = a.sinfo[b];
     if (si.n < 0) return;                                  // fatal sequence
     const bool pair = k < L;
     if (!pair && si.draw_row != L) return;                 // bonus row not needed
     const bool draw = si.draw_row == k;
+    const int v0 = s * sv;
+    const int nv = max(min(sv, R.nvec - v0), 0);
+    const char* prow = row_ptr(R, b, k) + (int64_t)v0 * 16;
+    const char* qrow = pair ? row_ptr(R, b, K + 1 + k) + (int64_t)v0 * 16 : nullptr;
+    uint4 rp[NV], rq[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        const int v = tid + u * WT;
+        rp[u] = neg_inf_vec<DT>(); rq[u] = neg_inf_vec<DT>();
+        if (v < nv) { rp[u] = ldg16(prow + (size_t)v * 16); if (pair) rq[u] = ldg16(qrow + (size_t)v * 16); }
+    }
     const float tau = tau_of(R, b);
     const float c = kLog2e / tau;
     const RowScale SP = row_scale(a.rstat[(int64_t)b * NR + k]);
     RowScale SQ; SQ.m = 0.f; SQ.frac = 0.f; SQ.inv = 0.f;
     if (pair) SQ = row_scale(a.rstat[(int64_t)b * NR + K + 1 + k]);
-    const int v0 = s * a.slice_vecs;
-    const int nv = max(min(a.slice_vecs, R.nvec - v0), 0);
-    const char* prow = row_ptr(R, b, k) + (int64_t)v0 * 16;
-    const char* qrow = pair ? row_ptr(R, b, K + 1 + k) + (int64_t)v0 * 16 : nullptr;
+    if ((v0 + nv) * VEC > R.V) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int gbase = (v0 + tid + u * WT) * VEC;
+            if (tid + u * WT < nv && gbase + VEC > R.V) { mask_tail<DT>(rp[u], R.V - gbase); mask_tail<DT>(rq[u], R.V - gbase); }
+        }
+    }
     float z0 = 0.f, z1 = 0.f, sqs = 0.f;
     double zd = 0.0;
-    for (int i0 = tid; i0 < nv; i0 += WT * 2) {
-        uint4 rp[2], rq[2];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int v = i0 + u * WT;
-            rp[u] = neg_inf_vec<DT>(); rq[u] = neg_inf_vec<DT>();
-            if (v < nv) {
-                rp[u] = ldg16(prow + (size_t)v * 16);
-                if (pair) rq[u] = ldg16(qrow + (size_t)v * 16);
-                const int gbase = (v0 + v) * VEC;
-                if (gbase + VEC > R.V) { mask_tail<DT>(rp[u], R.V - gbase); mask_tail<DT>(rq[u], R.V - gbase); }
-            }
-        }
+    for (int u = 0; u < NV; ++u) {
+        if (tid + u * WT < nv) {
+            float r[8];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            if (i0 + u * WT < nv) {
-                float r[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                residual_vec<DT>(rp[u], rq[u], pair, c, SP, SQ, r, draw ? &sqs : nullptr);
-                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-                if (u) z1 += vs; else z0 += vs;
-                if (draw) zd += (double)vs;
-            }
+            for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            residual_vec<DT>(rp[u], rq[u], pair, c, SP, SQ, r, draw ? &sqs : nullptr);
+            const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+            if (u & 1) z1 += vs; else z0 += vs;
+            if (draw) zd += (double)vs;
         }
     }
     float z = warp_sum(z0 + z1);
@@ -399,13 +419,13 @@ __device__ __forceinline__ void phase_p2(const WaveArgs& a, WaveShared& S, int b
         if (pair) {
             float zz = 0.f;
             for (int w = 0; w < WW; ++w) zz += S.redf[0][w];
-            a.zpart[((int64_t)b * K + k) * a.T + s] = zz;
+            a.zpart[((int64_t)b * K + k) * T2 + s] = zz;
         }
         if (draw) {
             double tot = 0.0; float sq = 0.f;
             for (int w = 0; w < WW; ++w) { tot += S.redd[w]; sq += S.redf[1][w]; }
             DPart d; d.tot = tot; d.sq = sq; d.pad = 0;
-            a.dpart[(int64_t)b * a.T + s] = d;
+            a.dpart[(int64_t)b * T2 + s] = d;
         }
     }
 }
@@ -416,7 +436,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
     constexpr int VEC = Elem<DT>::VEC;
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1, T = a.T;
+    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1, T = 2 * a.T, sv = a.slice_vecs >> 1;
     const SeqInfo si = a.sinfo[b];
     if (si.n < 0) return;
     // TV of every draft position: slice parts in slice order
@@ -450,8 +470,8 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
         const RowScale SP = row_scale(a.rstat[(int64_t)b * NR + k]);
         RowScale SQ; SQ.m = 0.f; SQ.frac = 0.f; SQ.inv = 0.f;
         if (pair) SQ = row_scale(a.rstat[(int64_t)b * NR + K + 1 + k]);
-        const int v0 = s * a.slice_vecs;
-        const int nv = max(min(a.slice_vecs, R.nvec - v0), 0);
+        const int v0 = s * sv;
+        const int nv = max(min(sv, R.nvec - v0), 0);
         const char* prow = row_ptr(R, b, k) + (int64_t)v0 * 16;
         const char* qrow = pair ? row_ptr(R, b, K + 1 + k) + (int64_t)v0 * 16 : nullptr;
         // per-vector residual mass, same arithmetic as phase P2
@@ -532,69 +552,73 @@ template <int DT>
 __global__ void __launch_bounds__(WT, 4) k_wave(const WaveArgs a) {
     __shared__ WaveShared S;
     const int tid = threadIdx.x;
-    const int K = a.r.K, T = a.T, NR = 2 * K + 1;
-    int next = 0;
+    const int K = a.r.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
+    // schedule constants (all tickets fit 31 bits).  Prologue: P1(0..lag).  Step w = 0 .. nw+1 holds
+    // A(w), P2(w-1), P1(w+lag+1), D(w-2): every phase sits one whole step behind the phase it needs.
+    const int B = a.r.B, WS = a.wave_seqs, LAG = a.lag;
+    const int c0 = NR * T, c2 = (K + 1) * T2;
+    auto N = [&](int w) { return w <= 0 ? 0 : min(B, w * WS); };                 // sequences in the first w waves
+    const int P = c0 * N(LAG + 1);
+    auto F = [&](int w) { return N(w) + c2 * N(w - 1) + c0 * (N(w + LAG + 1) - N(LAG + 1)) + N(w - 2); };
+    int next = 0, ntr = 0;
     if (tid == 0) next = atomicAdd(a.ticket, 1);
     for (;;) {
+        long long tr0 = 0, tr1 = 0, tr2 = 0;
         if (tid == 0) {
+            tr0 = clock64();
             const int t = next;
             S.ticket = t;
             if (t < a.ntickets) {
-                // closed-form schedule: P1(0..lag), then per wave w: A(w), P2(w), P1(w+lag+1), D(w-1); last D(nw-1)
-                const int B = a.r.B, WS = a.wave_seqs, LAG = a.lag;
-                auto N = [&](int w) { return w <= 0 ? 0 : min(B, w * WS); };           // sequences in the first w waves
-                const long long c0 = (long long)NR * T, c2 = (long long)(K + 1) * T;
-                const long long P = c0 * N(LAG + 1);
-                int ph, wv; long long off;
-                if (t < P) { ph = 0; wv = (int)(t / (c0 * WS)); off = t - c0 * N(wv); }
+                int ph, wv, off;
+                if (t < P) { ph = 0; wv = t / (c0 * WS); off = t - c0 * N(wv); }
                 else {
-                    auto F = [&](int w) { return (long long)N(w) * (1 + c2) + c0 * (N(w + LAG + 1) - N(LAG + 1)) + N(w - 1); };
-                    const long long tt = t - P;
-                    int lo = 0, hi = a.nwaves;
+                    const int tt = t - P;
+                    int lo = 0, hi = a.nwaves + 1;
                     while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (F(mid) <= tt) lo = mid; else hi = mid - 1; }
-                    const int w = lo;
-                    long long o2 = tt - F(w);
-                    const long long nA = N(w + 1) - N(w), n2 = nA * c2, n1 = c0 * (N(w + LAG + 2) - N(w + LAG + 1));
+                    const int w = lo, o2 = tt - F(w);
+                    const int nA = N(w + 1) - N(w), n2 = (N(w) - N(w - 1)) * c2, n1 = c0 * (N(w + LAG + 2) - N(w + LAG + 1));
                     if (o2 < nA) { ph = 1; wv = w; off = o2; }
-                    else if (o2 < nA + n2) { ph = 2; wv = w; off = o2 - nA; }
+                    else if (o2 < nA + n2) { ph = 2; wv = w - 1; off = o2 - nA; }
                     else if (o2 < nA + n2 + n1) { ph = 0; wv = w + LAG + 1; off = o2 - nA - n2; }
-                    else { ph = 3; wv = w - 1; off = o2 - nA - n2 - n1; }
+                    else { ph = 3; wv = w - 2; off = o2 - nA - n2 - n1; }
                 }
-                struct { int phase, wave; } sg = {ph, wv};
-                S.phase = ph; S.wave = wv; S.index = (int)off;
+                S.phase = ph; S.wave = wv; S.index = off;
                 next = atomicAdd(a.ticket, 1);
-                // dependencies: counters of the wave (almost always long satisfied)
-                const int w = sg.wave;
-                const int b0 = w * a.wave_seqs, ns = min(a.wave_seqs, a.r.B - b0);
+                // dependencies: completion counters of the wave (almost always long satisfied)
+                const int ns = N(wv + 1) - N(wv);
                 bool okw = true;
-                if (sg.phase == 1) okw = spin_ge(&a.p1done[w], ns * NR * T);
-                else if (sg.phase == 2) okw = spin_ge(&a.adone[w], ns);
-                else if (sg.phase == 3) okw = spin_ge(&a.p2done[w], ns * (K + 1) * T);
+                if (ph == 1) okw = spin_ge(&a.p1done[wv], ns * c0);
+                else if (ph == 2) okw = spin_ge(&a.adone[wv], ns);
+                else if (ph == 3) okw = spin_ge(&a.p2done[wv], ns * c2);
                 if (!okw) atomicExch(a.wait_failed, 1);
             }
         }
         __syncthreads();
         if (S.ticket >= a.ntickets) break;
+        if (tid == 0) tr1 = clock64();
         const int phase = S.phase, w = S.wave, idx = S.index;
-        const int b0 = w * a.wave_seqs;
+        const int b0 = w * WS;
+        int* done = nullptr;
         if (phase == 0) {
-            const int s = idx % T, r = (idx / T) % NR, b = b0 + idx / (T * NR);
+            const int s = idx % T, r = (idx / T) % NR, b = b0 + idx / c0;
             phase_p1<DT>(a, S, b, r, s);
-            __syncthreads();
-            if (tid == 0) { __threadfence(); atomicAdd(&a.p1done[w], 1); }
+            done = &a.p1done[w];
         } else if (phase == 1) {
             phase_a<DT>(a, S, b0 + idx);
-            __syncthreads();
-            if (tid == 0) { __threadfence(); atomicAdd(&a.adone[w], 1); }
+            done = &a.adone[w];
         } else if (phase == 2) {
-            const int s = idx % T, k = (idx / T) % (K + 1), b = b0 + idx / (T * (K + 1));
+            const int s = idx % T2, k = (idx / T2) % (K + 1), b = b0 + idx / c2;
             phase_p2<DT>(a, S, b, k, s);
-            __syncthreads();
-            if (tid == 0) { __threadfence(); atomicAdd(&a.p2done[w], 1); }
+            done = &a.p2done[w];
         } else {
             phase_d<DT>(a, S, b0 + idx);
         }
         __syncthreads();
+        // results consumed by later phases are written by thread 0: its release covers them
+        if (tid == 0 && done) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" :: "l"(done) : "memory");
+#ifdef BEBOP_TRACE
+        if (tid == 0 && a.trace && blockIdx.x == 7 && ntr < 60) { tr2 = clock64(); a.trace[ntr * 16 + 0] = phase + 1; a.trace[ntr * 16 + 1] = tr1 - tr0; a.trace[ntr * 16 + 2] = tr2 - tr1; a.trace[ntr * 16 + 3] = tr0; ntr++; }
+#endif
     }
 }
 
@@ -622,6 +646,9 @@ int wave_grid() {
 }
 
 }  // namespace
+
+long long* g_wave_trace = nullptr;
+void wave_set_trace(long long* p) { g_wave_trace = p; }
 
 bool wave_supported(const RowArgs& a) {
     const int T = (a.nvec + SLICE_VECS - 1) / SLICE_VECS;
@@ -651,11 +678,12 @@ cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.zpart = reinterpret_cast<float*>(w + wp.off_zpart);
     wa.dpart = reinterpret_cast<DPart*>(w + wp.off_dpart);
     wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
+    wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;
     // number of tickets: every phase of every wave
     {
         const long long NR = 2 * a.K + 1;
-        const long long total = (long long)a.B * (NR * wp.T + 1 + (long long)(a.K + 1) * wp.T + 1);
+        const long long total = (long long)a.B * (NR * wp.T + 1 + (long long)(a.K + 1) * 2 * wp.T + 1);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
         wa.lag = wp.lag;
