@@ -337,7 +337,14 @@ __device__ __forceinline__ void draw_stats_body(const RowArgs& a, const int* __r
         if (threadIdx.x == 0) {
             MSd t{shm[0], shs[0]};
             for (int i = 1; i < kThreads / 32; ++i) t = msd_merge(t, MSd{shm[i], shs[i]});
-            dstats[((int64_t)b * 2 + which) * nsplit_d + split] = make_double2(t.m, t.s);
+            // store the partial against an integer power of two, sum = s2 * 2^e, so that the merge of
+            // the slices is an exact rescaling (no exponentials)
+            double e = t.m, s2 = t.s;
+            if (t.m == t.m && t.m != INFINITY && t.m != -INFINITY) {
+                e = ceil(t.m * 1.4426950408889634);
+                s2 = t.s * exp(t.m - e * 0.6931471805599453);
+            }
+            dstats[((int64_t)b * 2 + which) * nsplit_d + split] = make_double2(e, s2);
         }
         __syncthreads();
     }
@@ -364,11 +371,22 @@ __global__ void __launch_bounds__(kThreads) k_draw_stats(RowArgs a, const int* _
 // Merge the fp64 partials of the stop row(s); returns status bits.
 __device__ __forceinline__ int draw_merge(const double2* dstats, int b, int nsplit_d, bool resid,
                                           DrawRow* d) {
+    // partials are (e, s2) with sum = s2 * 2^e, e an integer (or NaN / +-inf for a bad or empty slice)
     MSd P{-INFINITY, 0.0}, Q{-INFINITY, 0.0};
     const double2* sp = dstats + (int64_t)b * 2 * nsplit_d;
-    for (int s = 0; s < nsplit_d; ++s) {
-        P = msd_merge(P, MSd{sp[s].x, sp[s].y});
-        if (resid) Q = msd_merge(Q, MSd{sp[nsplit_d + s].x, sp[nsplit_d + s].y});
+    for (int w = 0; w < (resid ? 2 : 1); ++w) {
+        double em = -INFINITY;
+        bool nan = false;
+        for (int s = 0; s < nsplit_d; ++s) { const double e = sp[w * nsplit_d + s].x; if (e != e) nan = true; else em = fmax(em, e); }
+        double sum = 0.0;
+        if (!nan && em != INFINITY && em != -INFINITY)
+            for (int s = 0; s < nsplit_d; ++s) {
+                const double2 v = sp[w * nsplit_d + s];
+                if (v.x != -INFINITY) sum += scalbn(v.y, (int)fmax(v.x - em, -2000.0));
+            }
+        MSd& R_ = w ? Q : P;
+        R_.m = nan ? NAN : (em == INFINITY || em == -INFINITY ? em : em * 0.6931471805599453);
+        R_.s = (nan || em == INFINITY) ? NAN : sum;
     }
     int st = 0;
     if (P.m != P.m || P.m == INFINITY || P.s != P.s) st |= ST_NONFINITE;
