@@ -35,6 +35,27 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def ncu_traffic():
+    """DRAM bytes per launch of the wave kernel on the headline workload, from the committed ncu summary."""
+    try:
+        for ln in open(os.path.join(ROOT, "profiles", "k_wave_headline.md")):
+            if ln.startswith("traffic_bytes_per_launch"):
+                return int(ln.split("=")[1].split()[0])
+    except Exception:
+        pass
+    return None
+
+
+def roofline(alg_bytes, kern_ms, peak, peak_kind, headline):
+    """HBM roofline of the dominant kernel (k_wave): algorithmic bytes of one launch over its
+    CUDA-event duration measured inside the timed region."""
+    gbs = alg_bytes / (kern_ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+            "traffic": ncu_traffic() if headline else None, "peak_kind": "of " + peak_kind,
+            "kernel": "k_wave", "kernel_ms": kern_ms, "algorithmic_bytes_per_launch": alg_bytes,
+            "pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS}
+
+
 class ClockSampler:
     """Polls SM clock, power and throttle reasons through NVML (read-only)."""
 
@@ -134,7 +155,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "positions/s", "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "headline: B=%d K=3 V=151936 bf16 logits, tau=1 (oracle sample)"},
+        "config": {"workload": "headline: B=256 K=3 V=151936 bf16 logits, tau=1 (oracle sample)"},
         "cpu_baseline": {"value": val, "unit": "positions/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "positions/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -195,16 +216,31 @@ def run_ours(args):
         step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # events around the dominant kernel (the wave kernel) inside the timed region: the library records
+    # them on the launching stream; at most 256 steps carry a pair
+    stride = max(1, steps // 256)
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range((steps + stride - 1) // stride)]
+    for a_, b_ in pairs:            # a torch event owns a CUDA event only after its first record
+        a_.record(); b_.record()
+    torch.cuda.synchronize()
     t0 = time.perf_counter()
     e0.record()
-    for _ in range(steps):
+    for i in range(steps):
+        if i % stride == 0:
+            P.bebop_debug_set_timing_events(*pairs[i // stride])
+        else:
+            P.bebop_debug_set_timing_events(None, None)
         step()
     e1.record()
     barrier()
     t1 = time.perf_counter()
+    P.bebop_debug_set_timing_events(None, None)
     ms = e0.elapsed_time(e1)
+    kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
+    kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = int(os.environ.get("BEBOP_LAUNCHES_PER_CALL", "4"))
+    launches_per_call = 5 if args.path == 0 else 6      # wave, flag, 3 fp64 re-draw kernels | 6 general kernels
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))
@@ -253,26 +289,29 @@ def run_ours(args):
                                    "draft=target+N(0,1), per GPU" % B,
                        "global_batch": world * B, "positions_per_step": world * positions,
                        "l2": "inputs (%.0f MB per GPU) larger than the 126 MB L2; no flush" % (alg_bytes / 1e6),
-                       "draw": "fp64 inverse CDF at the stop row", "parallelism": "dp%d" % world},
+                       "draw": "fp32 inverse CDF kept when it clears the error bound, else re-drawn in fp64",
+                       "parallelism": "dp%d" % world},
             "clocks": clocks,
             "e2e": {"value": world * positions / e2e_s, "unit": "positions/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3},
             "gpu_launches": steps * launches_per_call,
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,
-            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                         "traffic": None, "peak_kind": "of " + peak_kind,
-                         "kernel": "whole call (all kernels of one bebop_verify)",
-                         "algorithmic_bytes_per_launch": alg_bytes},
+            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256 and args.path == 0),
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             cores = oracle.num_threads()
-            xc = {k: (v[:64].cpu() if hasattr(v, "cpu") else v) for k, v in x.items()}
-            _, probe = oracle_sample_rate(xc, min(8, B))
-            nseq = int(max(8, min(64, 8 * 12.0 / max(probe, 1e-3))))
-            val, dt = oracle_sample_rate(xc, nseq)
-            line["cpu_baseline"] = {"value": val, "unit": "positions/s", "cores": cores, "kind": "oracle",
-                                    "sample": "first %d of the step's 256 sequences, %.1f s" % (nseq, dt)}
+            nseq = min(64, B)
+            xc = {k: (v[:nseq].cpu() if hasattr(v, "cpu") else v) for k, v in x.items()}
+            oracle_sample_rate(xc, min(8, nseq))
+            reps, spent = 0, 0.0
+            while spent < 10.0 and reps < 1000:
+                _, dt = oracle_sample_rate(xc, nseq)
+                spent += dt
+                reps += 1
+            line["cpu_baseline"] = {"value": reps * nseq * K / spent, "unit": "positions/s", "cores": cores,
+                                    "kind": "oracle",
+                                    "sample": "first %d of the step's %d sequences, %d passes, %.1f s" % (nseq, B, reps, spent)}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -130,14 +130,17 @@ bebop_status_t bebop_greedy_verify(
 /*
  * Test and measurement hooks (no counterpart in the paper).
  * bebop_debug_force_general_path(1) makes bebop_verify use the split-row general
- * kernels even for shapes the fused cluster kernel takes (process-wide switch).
- * bebop_debug_fallback_offset returns the byte offset, inside the workspace of
- * this shape, of an int32 that after a bebop_verify call through the fused kernel
- * holds the number of sequences whose draw was re-done by the fp64 kernels.
+ * kernels even for shapes the wave kernel takes (process-wide switch; 0 restores).
+ * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
+ * shape, of an int32 that after a bebop_verify call holds the number of sequences
+ * whose draw was re-done by the fp64 kernels.
+ * bebop_debug_set_timing_events(start, stop): two cudaEvent_t handles that the next
+ * bebop_verify calls record around the wave kernel, on the caller's stream (NULL,
+ * NULL switches it off).
  */
 void bebop_debug_force_general_path(int on);
-int bebop_debug_fused_clusters(bebop_dtype_t dt);   /* co-resident clusters the fused kernel gets on this device */
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
+void bebop_debug_set_timing_events(void* start, void* stop);
 
 /* Static, host-side, human-readable name of a status code. */
 const char* bebop_status_string(bebop_status_t status);

@@ -47,6 +47,8 @@ def load_library():
     lib.bebop_greedy_verify.argtypes = [vp, i64, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     lib.bebop_debug_force_general_path.restype = None
     lib.bebop_debug_force_general_path.argtypes = [i32]
+    lib.bebop_debug_set_timing_events.restype = None
+    lib.bebop_debug_set_timing_events.argtypes = [vp, vp]
     lib.bebop_debug_fallback_offset.restype = sz
     lib.bebop_debug_fallback_offset.argtypes = [i32, i32, i32, i32]
     lib.bebop_status_string.restype = C.c_char_p
@@ -89,6 +91,15 @@ def _rows(t: torch.Tensor, ndim: int):
 
 def bebop_debug_force_general_path(on: bool) -> None:
     load_library().bebop_debug_force_general_path(int(on))
+
+
+def bebop_debug_set_timing_events(start, stop) -> None:
+    """torch.cuda.Event pair (enable_timing=True, already recorded once) bracketing the wave kernel; None, None = off."""
+    lib = load_library()
+    if start is None:
+        lib.bebop_debug_set_timing_events(None, None)
+    else:
+        lib.bebop_debug_set_timing_events(C.c_void_p(start.cuda_event), C.c_void_p(stop.cuda_event))
 
 
 def bebop_debug_fallback_offset(B: int, K: int, V: int, dt: int) -> int:

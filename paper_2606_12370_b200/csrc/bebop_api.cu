@@ -9,7 +9,7 @@ namespace {
 
 // Test hook: route bebop_verify through the general (split-row) path even where the fused
 // kernel applies, so that both paths are covered by the parity tests.
-int g_path = 0;   // 0: ring kernel where it applies, 1: general kernels, 2: lockstep fused kernel, 3: register streaming kernel
+int g_path = 0;   // 0: wave kernel where it applies, otherwise the general kernels
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -96,14 +96,6 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     bool launched = false;
     if (g_path == 0 && wave_supported(a))
         e = wave_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    else if (g_path == 5 && tile_supported(a))
-        e = tile_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    else if (g_path == 4 && ring_supported(a))
-        e = ring_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    else if (g_path == 3 && stream_supported(a))
-        e = stream_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    else if (g_path == 2 && fused_supported(a))
-        e = fused_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
     if (e == cudaSuccess && !launched) e = general_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
@@ -151,9 +143,9 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
 
 void bebop_debug_force_general_path(int on) { g_path = on; }
 
-void bebop_debug_set_trace(void* p) { fused_set_trace(static_cast<long long*>(p)); stream_set_trace(static_cast<long long*>(p)); ring_set_trace(static_cast<long long*>(p)); wave_set_trace(static_cast<long long*>(p)); }
+void bebop_debug_set_trace(void* p) { wave_set_trace(static_cast<long long*>(p)); }
 
-int bebop_debug_fused_clusters(bebop_dtype_t dt) { return ring_max_clusters((int)dt); }
+void bebop_debug_set_timing_events(void* start, void* stop) { wave_set_events(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop)); }
 
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
     if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;

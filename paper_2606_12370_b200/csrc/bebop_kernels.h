@@ -44,40 +44,10 @@ cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft
 cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
                               const int* list, const int* count, cudaStream_t stream);
 
-// Fused single-read cluster kernel (bebop_fused.cu).  fused_verify sets *launched = false and
-// does nothing when the shape or the device cannot take it; the caller then uses general_verify.
-bool fused_supported(const RowArgs& a);
-int fused_max_clusters(int dt);
-void fused_set_trace(long long* p);
-cudaError_t fused_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                         cudaStream_t stream, bool* launched);
-
-// Streaming cluster kernel (bebop_stream.cu): same contract as fused_verify.
-bool stream_supported(const RowArgs& a);
-int stream_max_clusters(int dt);
-void stream_set_trace(long long* p);
-cudaError_t stream_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                          const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                          cudaStream_t stream, bool* launched);
-
-// Ring kernel (bebop_ring.cu): tensor-memory rings, same contract as fused_verify.
-bool ring_supported(const RowArgs& a);
-int ring_max_clusters(int dt);
-void ring_set_trace(long long* p);
-cudaError_t ring_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                        cudaStream_t stream, bool* launched);
-
-// Tile kernel (bebop_tile.cu): small vocabulary tiles, one CTA per tile; same contract.
-bool tile_supported(const RowArgs& a);
-cudaError_t tile_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                        cudaStream_t stream, bool* launched);
-
 // Wave kernel (bebop_wave.cu): persistent, ticket-scheduled, phases decoupled; same contract.
 bool wave_supported(const RowArgs& a);
 void wave_set_trace(long long* p);
+void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the wave kernel of the next calls (nullptr: off)
 cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);

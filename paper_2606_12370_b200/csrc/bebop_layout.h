@@ -30,26 +30,11 @@ struct Plan {
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
     size_t off_fb;      // int [1 + B]: count and list of sequences whose draw goes to fp64
-    size_t off_tile;    // workspace of the tile kernel
     size_t off_wave;    // workspace of the wave kernel
     size_t total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-
-constexpr int kTileVecs = 640;   // 16-byte vectors per row and tile of the tile kernel, at most
-
-// Workspace of the tile kernel: ticket + flags, per-row and per-sequence counters (zeroed at every
-// call), then the per-tile partials (32 B), Z parts (4 B) and residual masses (16 B).
-static inline size_t tile_ws_zero_bytes(int B, int K) {
-    const size_t rows = (size_t)B * (K + 1);
-    return 256 + 3 * align256(sizeof(int) * rows) + 4 * align256(sizeof(int) * (size_t)B);
-}
-static inline size_t tile_ws_bytes(int B, int K, int nvec) {
-    const size_t rows = (size_t)B * (K + 1);
-    const size_t T = (size_t)(nvec + kTileVecs - 1) / kTileVecs;
-    return tile_ws_zero_bytes(B, K) + align256(32 * rows * T) + align256(4 * rows * T) + align256(16 * (size_t)B * T);
-}
 
 static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
     (void)dt;
@@ -105,7 +90,6 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
-    p.off_tile = o;   o = align256(o + tile_ws_bytes(B, K, p.nvec));
     p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
     p.total = o;
     return p;

@@ -649,6 +649,8 @@ int wave_grid() {
 
 long long* g_wave_trace = nullptr;
 void wave_set_trace(long long* p) { g_wave_trace = p; }
+cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+void wave_set_events(cudaEvent_t start, cudaEvent_t stop) { g_ev_start = start; g_ev_stop = stop; }
 
 bool wave_supported(const RowArgs& a) {
     const int T = (a.nvec + SLICE_VECS - 1) / SLICE_VECS;
@@ -693,9 +695,11 @@ cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     e = cudaMemsetAsync(wa.fb_count, 0, sizeof(int), stream);
     if (e != cudaSuccess) return e;
     const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
+    if (g_ev_start) cudaEventRecord(g_ev_start, stream);
     if (a.dt == 0) k_wave<0><<<grid, WT, 0, stream>>>(wa);
     else k_wave<1><<<grid, WT, 0, stream>>>(wa);
     e = cudaGetLastError();
+    if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;
     k_wave_flag<<<(a.B + 255) / 256, 256, 0, stream>>>(wa.wait_failed, o.row_status, a.B);
     e = cudaGetLastError();
