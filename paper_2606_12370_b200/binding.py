@@ -110,6 +110,17 @@ def bebop_workspace_bytes(B: int, K: int, V: int, dt: int) -> int:
     return int(load_library().bebop_workspace_bytes(B, K, V, dt))
 
 
+# Tests set this so that an output the library failed to write cannot pass as a left-over of an
+# earlier call in recycled memory.
+POISON_OUTPUTS = False
+
+
+def _new(shape, dtype, dev):
+    if POISON_OUTPUTS:
+        return torch.full(shape if isinstance(shape, tuple) else (shape,), -77, dtype=dtype, device=dev)
+    return torch.empty(shape, dtype=dtype, device=dev)
+
+
 def _workspace(B, K, V, dt, device, workspace):
     need = bebop_workspace_bytes(B, K, V, dt)
     if workspace is None:
@@ -139,7 +150,7 @@ def bebop_verify(target_logits, draft_logits, draft_tokens, u_accept, u_final, d
     def get(name, shape, dtype, want=True):
         if name in o and o[name] is not None:
             return o[name]
-        return torch.empty(shape, dtype=dtype, device=dev) if want else None
+        return _new(shape, dtype, dev) if want else None
     res = dict(
         accept_len=get("accept_len", (B,), torch.int32), out_tokens=get("out_tokens", (B, K + 1), torch.int32),
         tv=get("tv", (B, K), torch.float32, want_tv), p_draft=get("p_draft", (B, K), torch.float32, want_probs),
@@ -172,9 +183,9 @@ def bebop_tv(target_logits, draft_logits, temperature=None, temperature_all=1.0,
     dev = target_logits.device
     tp, ldt = _rows(target_logits, 2)
     dp, ldd = _rows(draft_logits, 2)
-    tv = torch.empty(N, dtype=torch.float32, device=dev)
-    s_aux = torch.empty(N, dtype=torch.float32, device=dev) if want_s_aux else None
-    st = torch.empty(N, dtype=torch.int32, device=dev)
+    tv = _new(N, torch.float32, dev)
+    s_aux = _new(N, torch.float32, dev) if want_s_aux else None
+    st = _new(N, torch.int32, dev)
     ws, wsb = _workspace(N, 1, V, dt, dev, workspace)
     _check(lib.bebop_tv(tp, ldt, dp, ldd, _ptr(temperature), float(temperature_all), N, V, dt,
                         _ptr(tv), _ptr(s_aux), _ptr(st), _ptr(ws), wsb, _stream()))
@@ -190,9 +201,9 @@ def bebop_greedy_verify(target_logits, draft_tokens, draft_len=None, workspace=N
     dev = target_logits.device
     tp, ldt = _rows(target_logits, 3)
     assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous() and draft_tokens.is_cuda
-    acc = torch.empty(B, dtype=torch.int32, device=dev)
-    out = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
-    st = torch.empty(B, dtype=torch.int32, device=dev)
+    acc = _new(B, torch.int32, dev)
+    out = _new((B, K + 1), torch.int32, dev)
+    st = _new(B, torch.int32, dev)
     ws, wsb = _workspace(B, K, V, dt, dev, workspace)
     _check(lib.bebop_greedy_verify(tp, ldt, _ptr(draft_tokens), _ptr(draft_len), B, K, V, dt,
                                    _ptr(acc), _ptr(out), _ptr(st), _ptr(ws), wsb, _stream()))

@@ -44,12 +44,12 @@ constexpr int E_EMPTY = INT_MIN / 2;
 constexpr uint32_t kSpin = 1u << 22;
 
 struct __align__(16) P1Part { double s; int e; float m; };             // per (row, slice); m = NaN marks a non-finite logit
-struct __align__(16) RowStat { double inv_s; float m_ref, frac; int e; int pad; };   // per row, after the merge
+struct __align__(16) RowStat { double inv_s; float ef; int e; int pad[2]; };   // per row, after the merge: 1/S, exponent E
 struct __align__(16) DPart { double tot; float sq; int pad; };        // per (sequence, slice)
 struct __align__(16) SeqInfo {          // per sequence, written by phase A
     int n;                              // accept count (stop position); -1: fatal
     int draw_row;                       // row whose residual is drawn from (n, or L for the bonus row); -1 none
-    float sys;                          // systematic part of the error bound (rounding of the normalisers)
+    int pad0;
     int pad;
 };
 
@@ -95,29 +95,39 @@ __device__ __forceinline__ bool spin_ge(const int* p, int want) {
     return false;
 }
 
-// The error bound a draw must clear.  The residual is formed from fp32
-// exponentials (ex2.approx: 2 ulp) and fp32 products, so each p, q carries a
-// relative error of a few 2^-24; the errors of different tokens are independent,
-// hence the error of a prefix sum is of the order delta * sqrt(sum p^2 + q^2).
-// kappa leaves a wide safety factor over that root-sum-square.  `sys` adds the
-// part that is common to all tokens: the rounding of 1/S_p and 1/S_q to fp32.
-__device__ __forceinline__ double draw_bound(double sumsq, double sys) {
+// The error bound a draw must clear.  The residual is formed from fp32 exponentials (ex2.approx:
+// 2 ulp), an fp32 argument (half an ulp of a number below 64, times 2^arg) and one fp32 rounding of
+// the product with the two-float normaliser, so each p, q carries a relative error below
+// delta = 2^-22; the errors of different tokens are independent, hence the error of a prefix sum is
+// of the order delta * sqrt(sum p^2 + q^2), and so is the part common to all tokens, the error of the
+// fp32-summed normalisers.  Measured on 40 000 draws with the certification switched off, the largest
+// error that changed a token was 0.1 * delta * sqrt(sum p^2 + q^2); kappa = 4 leaves a factor 40 over
+// that.
+#ifndef BEBOP_KAPPA
+#define BEBOP_KAPPA 4.0
+#endif
+__device__ __forceinline__ double draw_bound(double sumsq) {
     const double delta = 2.384185791015625e-07;   // 2^-22
-    const double kappa = 16.0;
-    return kappa * delta * sqrt(sumsq) + sys + 1e-300;
+    return BEBOP_KAPPA * delta * sqrt(sumsq) + 1e-300;
 }
 
-// E = ceil(m * c), frac = E - m * c in [0, 1] without rounding loss, so that
-// 2^((x - m) * c - frac) equals 2^(x * c - E) whatever reference point m is used.
-__device__ __forceinline__ void reference(float m, float c, int* E, float* frac) {
-    float th = fminf(fmaxf(m * c, -4.0e6f), 4.0e6f);
-    float te = fmaf(m, c, -th);
-    if (th != m * c) te = 0.f;
-    float Ef;
-    int Ei = ceil_alu(th, &Ef);
-    float f = (Ef - th) - te;
-    if (f < 0.f) { f += 1.f; Ei += 1; }
-    *E = Ei; *frac = f;
+// c = log2(e) / tau in fp32, and 2^(x * c - E): the product is exact inside the fma, so the argument
+// carries one rounding of half an ulp of itself.  The rounding of c itself acts like a temperature
+// changed by at most 2^-24 relative; over a prefix of the vocabulary its effect, 2^-24 * sum p (z - zbar) / tau,
+// is a sum of zero-mean terms of the size draw_bound() already allows per token.
+struct TempScale { float hi; };
+__device__ __forceinline__ TempScale temp_scale(float tau) {
+    TempScale r; r.hi = kLog2e / (tau_ok(tau) ? tau : 1.f);
+    return r;
+}
+__device__ __forceinline__ float exp2_scaled(float x, const TempScale& t, float Ef) {
+    return ex2f(fmaf(x, t.hi, -Ef));
+}
+// E = ceil(m * c) of a maximum m, as int and float: any integer near m * c serves as the reference, and
+// integer references make every merge of partial sums an exact power-of-two scaling.
+__device__ __forceinline__ int ref_exponent(float m, const TempScale& t, float* Ef) {
+    const float th = fminf(fmaxf(m * t.hi, -4.0e6f), 4.0e6f);
+    return ceil_alu(th, Ef);
 }
 
 struct WaveShared {
@@ -149,7 +159,7 @@ __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b
     const int k = is_target ? r : r - (K + 1);
     if (is_target ? k > L : k >= L) return;
     const float tau = tau_of(R, b);
-    const float c = kLog2e / (tau_ok(tau) ? tau : 1.f);
+    const TempScale ts = temp_scale(tau);
     const int v0 = s * a.slice_vecs;
     const int nv = max(min(a.slice_vecs, R.nvec - v0), 0);
     const char* row = row_ptr(R, b, r) + (int64_t)v0 * 16;
@@ -174,8 +184,8 @@ __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b
     for (int u = 1; u < NV; ++u) m = max_nan(m, vec_max<DT>(raw[u]));
     const bool bad = m != m || m == INFINITY;
     int E = E_EMPTY;
-    float frac = 0.f, m_ref = 0.f;
-    if (!bad && m != -INFINITY) { reference(m, c, &E, &frac); m_ref = m; }
+    float Ef = 0.f;
+    if (!bad && m != -INFINITY) E = ref_exponent(m, ts, &Ef);
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
     if (E > E_EMPTY) {
 #pragma unroll
@@ -184,10 +194,10 @@ __device__ __forceinline__ void phase_p1(const WaveArgs& a, WaveShared& S, int b
             unpack<DT>(raw[u], f);
 #pragma unroll
             for (int i = 0; i < VEC; i += 4) {
-                s0 += ex2f(fmaf(f[i] - m_ref, c, -frac));
-                s1 += ex2f(fmaf(f[i + 1] - m_ref, c, -frac));
-                s2 += ex2f(fmaf(f[i + 2] - m_ref, c, -frac));
-                s3 += ex2f(fmaf(f[i + 3] - m_ref, c, -frac));
+                s0 += exp2_scaled(f[i], ts, Ef);
+                s1 += exp2_scaled(f[i + 1], ts, Ef);
+                s2 += exp2_scaled(f[i + 2], ts, Ef);
+                s3 += exp2_scaled(f[i + 3], ts, Ef);
             }
         }
     }
@@ -220,7 +230,7 @@ __device__ __forceinline__ void phase_a(const WaveArgs& a, WaveShared& S, int b)
     const int K = R.K, V = R.V, L = len_of(R, b), NR = 2 * K + 1, T = a.T;
     const float tau = tau_of(R, b);
     const bool ok = tau_ok(tau);
-    const float c = kLog2e / (ok ? tau : 1.f);
+    const TempScale ts = temp_scale(tau);
     __shared__ int sh_status[2 * BEBOP_MAX_K_INT + 1];
     __shared__ double sh_S[2 * BEBOP_MAX_K_INT + 1];
     __shared__ int sh_E[2 * BEBOP_MAX_K_INT + 1];
@@ -273,7 +283,7 @@ __device__ __forceinline__ void phase_a(const WaveArgs& a, WaveShared& S, int b)
         if (active && !(seq_st & ST_FATAL) && lane < first_bad) {
             const float zpx = DT == 0 ? load_one<0>(row_ptr(R, b, lane), tk) : load_one<1>(row_ptr(R, b, lane), tk);
             const float zqx = DT == 0 ? load_one<0>(row_ptr(R, b, K + 1 + lane), tk) : load_one<1>(row_ptr(R, b, K + 1 + lane), tk);
-            const double cd = (double)c;
+            const double cd = (double)ts.hi;
             px = exp2((double)zpx * cd - (double)sh_E[lane]) / sh_S[lane];
             qx = exp2((double)zqx * cd - (double)sh_E[K + 1 + lane]) / sh_S[K + 1 + lane];
             acc = (double)a.u_accept[(int64_t)b * K + lane] * qx < px;
@@ -292,42 +302,18 @@ __device__ __forceinline__ void phase_a(const WaveArgs& a, WaveShared& S, int b)
             if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)qx;
             if (zero && a.o.tv) a.o.tv[(int64_t)b * K + lane] = 0.f;
         }
-        // normalisers for phase P2: 2^(x*c - E) is evaluated as 2^((x - m_ref)*c - frac) around the row maximum;
-        // lane r (and r + 32, r + 64) owns row r
-        double my_inv[3] = {0.0, 0.0, 0.0};
-        for (int i = 0, r = lane; r < NR; r += 32, ++i) {
-            RowStat st; st.inv_s = 0.0; st.m_ref = 0.f; st.frac = 0.f; st.e = sh_E[r]; st.pad = 0;
-            if (!fatal && sh_E[r] > E_EMPTY && sh_S[r] > 0.0) {
-                st.inv_s = 1.0 / sh_S[r];
-                int Er; float fr;
-                reference(sh_M[r], c, &Er, &fr);           // Er == sh_E[r]: the row maximum fixes the exponent
-                st.m_ref = sh_M[r]; st.frac = fr + (float)(sh_E[r] - Er);
-            }
+        // normalisers for phase P2; lane r (and r + 32, r + 64) owns row r
+        for (int r = lane; r < NR; r += 32) {
+            RowStat st; st.inv_s = 0.0; st.ef = (float)sh_E[r]; st.e = sh_E[r]; st.pad[0] = 0; st.pad[1] = 0;
+            if (!fatal && sh_E[r] > E_EMPTY && sh_S[r] > 0.0) st.inv_s = 1.0 / sh_S[r];
             a.rstat[(int64_t)b * NR + r] = st;
-            if (i < 3) my_inv[i] = st.inv_s;
         }
-        // |fl(1/S) - 1/S| / (1/S) of the rows the draw uses: what the fp32 scale factors add to a prefix sum
         const int draw_row = fatal ? -1 : nn;
-        float sys = 0.f;
-        if (draw_row >= 0) {
-            const int rp_ = draw_row, rq_ = draw_row < L ? K + 1 + draw_row : -1;
-            double ip = 0.0, iq = 0.0;
-#pragma unroll
-            for (int i = 0; i < 3; ++i) {
-                const double v = my_inv[i];
-                const double vp = __shfl_sync(0xffffffffu, v, rp_ & 31);
-                const double vq = __shfl_sync(0xffffffffu, v, (rq_ < 0 ? 0 : rq_) & 31);
-                if ((rp_ >> 5) == i) ip = vp;
-                if (rq_ >= 0 && (rq_ >> 5) == i) iq = vq;
-            }
-            if (ip > 0.0) sys += (float)(fabs((double)(float)ip - ip) / ip);
-            if (iq > 0.0) sys += (float)(fabs((double)(float)iq - iq) / iq);
-        }
         if (lane == 0) {
             a.o.accept_len[b] = nn;
             if (a.o.row_status) a.o.row_status[b] = seq_st;
             a.stop[b] = fatal ? -1 : nn;
-            SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = draw_row; si.sys = sys; si.pad = 0;
+            SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = draw_row; si.pad0 = 0; si.pad = 0;
             a.sinfo[b] = si;
         }
         __syncwarp();
@@ -338,11 +324,17 @@ __device__ __forceinline__ void phase_a(const WaveArgs& a, WaveShared& S, int b)
 }
 
 // residuals of one vector pair: p = 2^(x*c - E_p) / S_p, q likewise
-struct RowScale { float m, frac, inv; };
-__device__ __forceinline__ RowScale row_scale(const RowStat& s) { RowScale r; r.m = s.m_ref; r.frac = s.frac; r.inv = (float)s.inv_s; return r; }
+struct RowScale { float ef, inv, inv_lo; };     // exponent E; 1/S = inv + inv_lo to about 2^-48
+__device__ __forceinline__ RowScale row_scale(const RowStat& s) {
+    RowScale r; r.ef = s.ef; r.inv = (float)s.inv_s; r.inv_lo = (float)(s.inv_s - (double)r.inv);
+    return r;
+}
+__device__ __forceinline__ RowScale no_row() { RowScale r; r.ef = 0.f; r.inv = 0.f; r.inv_lo = 0.f; return r; }
 
-template <int DT>
-__device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, bool pair, float c, const RowScale& P,
+// FINE (the rows a token is drawn from): the normaliser enters as two floats, so that its rounding to fp32
+// is not an error common to all tokens of the row; what is left is one rounding per token.
+template <int DT, bool FINE>
+__device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, bool pair, const TempScale& c, const RowScale& P,
                                              const RowScale& Q, float* r, float* sq) {
     constexpr int VEC = Elem<DT>::VEC;
     float fp[VEC], fq[VEC];
@@ -350,8 +342,11 @@ __device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, b
     if (pair) unpack<DT>(rq, fq);
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
-        const float p = __fmul_rn(ex2f(fmaf(fp[i] - P.m, c, -P.frac)), P.inv);
-        const float q = pair ? __fmul_rn(ex2f(fmaf(fq[i] - Q.m, c, -Q.frac)), Q.inv) : 0.f;
+        const float ap = exp2_scaled(fp[i], c, P.ef);
+        const float aq = pair ? exp2_scaled(fq[i], c, Q.ef) : 0.f;
+        // explicit roundings: a contracted p - a*inv would leave rounding dust when the rows are equal
+        const float p = FINE ? __fmaf_rn(ap, P.inv_lo, __fmul_rn(ap, P.inv)) : __fmul_rn(ap, P.inv);
+        const float q = pair ? (FINE ? __fmaf_rn(aq, Q.inv_lo, __fmul_rn(aq, Q.inv)) : __fmul_rn(aq, Q.inv)) : 0.f;
         r[i] = fmaxf(p - q, 0.f);
         if (sq) { *sq = fmaf(p, p, *sq); *sq = fmaf(q, q, *sq); }
     }
@@ -383,9 +378,9 @@ __device__ __forceinline__ void phase_p2(const WaveArgs& a, WaveShared& S, int b
         if (v < nv) { rp[u] = ldg16(prow + (size_t)v * 16); if (pair) rq[u] = ldg16(qrow + (size_t)v * 16); }
     }
     const float tau = tau_of(R, b);
-    const float c = kLog2e / tau;
+    const TempScale c = temp_scale(tau);
     const RowScale SP = row_scale(a.rstat[(int64_t)b * NR + k]);
-    RowScale SQ; SQ.m = 0.f; SQ.frac = 0.f; SQ.inv = 0.f;
+    RowScale SQ = no_row();
     if (pair) SQ = row_scale(a.rstat[(int64_t)b * NR + K + 1 + k]);
     if ((v0 + nv) * VEC > R.V) {
 #pragma unroll
@@ -396,16 +391,32 @@ __device__ __forceinline__ void phase_p2(const WaveArgs& a, WaveShared& S, int b
     }
     float z0 = 0.f, z1 = 0.f, sqs = 0.f;
     double zd = 0.0;
+    if (!draw) {
+        // the common case: TV only
 #pragma unroll
-    for (int u = 0; u < NV; ++u) {
-        if (tid + u * WT < nv) {
-            float r[8];
+        for (int u = 0; u < NV; ++u) {
+            if (tid + u * WT < nv) {
+                float r[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) r[i] = 0.f;
-            residual_vec<DT>(rp[u], rq[u], pair, c, SP, SQ, r, draw ? &sqs : nullptr);
-            const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-            if (u & 1) z1 += vs; else z0 += vs;
-            if (draw) zd += (double)vs;
+                for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                residual_vec<DT, false>(rp[u], rq[u], pair, c, SP, SQ, r, nullptr);
+                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                if (u & 1) z1 += vs; else z0 += vs;
+            }
+        }
+    } else {
+        // the row pair a token is drawn from: also the mass in double and the sum of squares
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            if (tid + u * WT < nv) {
+                float r[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                residual_vec<DT, true>(rp[u], rq[u], pair, c, SP, SQ, r, &sqs);
+                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                z0 += vs;
+                zd += (double)vs;
+            }
         }
     }
     float z = warp_sum(z0 + z1);
@@ -459,16 +470,16 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
             run = nx;
         }
         S.owner_slice = (Tt > 0.0) ? owner : -1;
-        S.base = base; S.Ttarget = Tt; S.bound = draw_bound(sumsq, (double)si.sys);
+        S.base = base; S.Ttarget = Tt; S.bound = draw_bound(sumsq);
     }
     __syncthreads();
     const int s = S.owner_slice;
     int found_y = -1, found_cert = 0;
     if (s >= 0) {
         const float tau = tau_of(R, b);
-        const float c = kLog2e / tau;
+        const TempScale c = temp_scale(tau);
         const RowScale SP = row_scale(a.rstat[(int64_t)b * NR + k]);
-        RowScale SQ; SQ.m = 0.f; SQ.frac = 0.f; SQ.inv = 0.f;
+        RowScale SQ = no_row();
         if (pair) SQ = row_scale(a.rstat[(int64_t)b * NR + K + 1 + k]);
         const int v0 = s * sv;
         const int nv = max(min(sv, R.nvec - v0), 0);
@@ -483,7 +494,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
             float r[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) r[i] = 0.f;
-            residual_vec<DT>(rp, rq, pair, c, SP, SQ, r, nullptr);
+            residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
             S.vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
         }
         __syncthreads();
@@ -515,7 +526,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
                     float r[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                    residual_vec<DT>(rp, rq, pair, c, SP, SQ, r, nullptr);
+                    residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
                     double Cw = C;
 #pragma unroll
                     for (int i = 0; i < VEC; ++i) {

@@ -24,3 +24,17 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _poison_outputs():
+    """Outputs start from a sentinel: nothing passes on values left in recycled device memory."""
+    try:
+        import paper_2606_12370_b200.binding as binding
+    except Exception:
+        yield
+        return
+    old = binding.POISON_OUTPUTS
+    binding.POISON_OUTPUTS = True
+    yield
+    binding.POISON_OUTPUTS = old
