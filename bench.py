@@ -240,7 +240,7 @@ def run_ours(args):
     kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
     kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = 5 if args.path == 0 else 6      # wave, flag, 3 fp64 re-draw kernels | 6 general kernels
+    launches_per_call = 4 if args.path == 0 else 6      # wave, flag, 2 fp64 re-draw kernels | 6 general kernels
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))

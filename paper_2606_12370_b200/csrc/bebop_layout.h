@@ -12,7 +12,8 @@ struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
     int wave_seqs, nwaves; // sequences per wave, waves
     int lag;               // waves of stats work scheduled between a phase and the phase it depends on
-    size_t off_p1done, off_adone, off_p2done, zero_bytes;
+    size_t off_p1done, off_adone, off_p2done, off_xdone, zero_bytes;
+    size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
     size_t off_part, off_rstat, off_zpart, off_dpart, off_sinfo, total;
 };
 
@@ -53,7 +54,10 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
     w.off_p1done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
     w.off_adone = o;  o += align256(sizeof(int) * (size_t)w.nwaves);
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
+    w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
     w.zero_bytes = o;
+    w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);
+    w.off_xmass = o;  o += align256(8 * (size_t)B * 4 * w.T * 8);
     w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
     w.off_rstat = o;  o += align256(32 * (size_t)B * NR);
     w.off_zpart = o;  o += align256(4 * (size_t)B * (K > 0 ? K : 1) * 2 * w.T);
