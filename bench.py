@@ -270,10 +270,8 @@ def run_ours(args):
     d2h = sum(host_out[k].numel() * host_out[k].element_size() for k in host_out)
 
     # max over ranks
-    if dist is not None:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
+    from paper_2606_12370_b200.shard import max_over_ranks
+    ms, e2e_s = max_over_ranks([ms, e2e_s], dist, dev)
     sampler.stop()
 
     if rank == 0:

@@ -571,12 +571,15 @@ __global__ void __launch_bounds__(WT, 4) k_wave(const WaveArgs a) {
     auto N = [&](int w) { return w <= 0 ? 0 : min(B, w * WS); };                 // sequences in the first w waves
     const int P = c0 * N(LAG + 1);
     auto F = [&](int w) { return N(w) + c2 * N(w - 1) + c0 * (N(w + LAG + 1) - N(LAG + 1)) + N(w - 2); };
-    int next = 0, ntr = 0;
+    int next = 0;
     if (tid == 0) next = atomicAdd(a.ticket, 1);
     for (;;) {
-        long long tr0 = 0, tr1 = 0, tr2 = 0;
+        long long tr0 = 0, tr1 = 0, trd = 0, trs = 0;
+        (void)tr1; (void)trd; (void)trs;
         if (tid == 0) {
+#ifdef BEBOP_TRACE
             tr0 = clock64();
+#endif
             const int t = next;
             S.ticket = t;
             if (t < a.ntickets) {
@@ -595,6 +598,9 @@ __global__ void __launch_bounds__(WT, 4) k_wave(const WaveArgs a) {
                 }
                 S.phase = ph; S.wave = wv; S.index = off;
                 next = atomicAdd(a.ticket, 1);
+#ifdef BEBOP_TRACE
+                trd = clock64();
+#endif
                 // dependencies: completion counters of the wave (almost always long satisfied)
                 const int ns = N(wv + 1) - N(wv);
                 bool okw = true;
@@ -602,11 +608,16 @@ __global__ void __launch_bounds__(WT, 4) k_wave(const WaveArgs a) {
                 else if (ph == 2) okw = spin_ge(&a.adone[wv], ns);
                 else if (ph == 3) okw = spin_ge(&a.p2done[wv], ns * c2);
                 if (!okw) atomicExch(a.wait_failed, 1);
+#ifdef BEBOP_TRACE
+                trs = clock64();
+#endif
             }
         }
         __syncthreads();
         if (S.ticket >= a.ntickets) break;
+#ifdef BEBOP_TRACE
         if (tid == 0) tr1 = clock64();
+#endif
         const int phase = S.phase, w = S.wave, idx = S.index;
         const int b0 = w * WS;
         int* done = nullptr;
@@ -628,7 +639,14 @@ __global__ void __launch_bounds__(WT, 4) k_wave(const WaveArgs a) {
         // results consumed by later phases are written by thread 0: its release covers them
         if (tid == 0 && done) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" :: "l"(done) : "memory");
 #ifdef BEBOP_TRACE
-        if (tid == 0 && a.trace && blockIdx.x == 7 && ntr < 60) { tr2 = clock64(); a.trace[ntr * 16 + 0] = phase + 1; a.trace[ntr * 16 + 1] = tr1 - tr0; a.trace[ntr * 16 + 2] = tr2 - tr1; a.trace[ntr * 16 + 3] = tr0; ntr++; }
+        if (tid == 0 && a.trace) {
+            // per phase: cycles in ticket decode, dependency wait, barrier, task; task count
+            const long long tr2 = clock64();
+            unsigned long long* tq = reinterpret_cast<unsigned long long*>(a.trace) + phase * 8;
+            atomicAdd(tq + 0, (unsigned long long)(trd - tr0)); atomicAdd(tq + 1, (unsigned long long)(trs - trd));
+            atomicAdd(tq + 2, (unsigned long long)(tr1 - trs)); atomicAdd(tq + 3, (unsigned long long)(tr2 - tr1));
+            atomicAdd(tq + 4, 1ull);
+        }
 #endif
     }
 }
