@@ -44,7 +44,8 @@ typedef enum {
     BEBOP_ERR_WORKSPACE = 5,
     BEBOP_ERR_TEMPERATURE = 6,
     BEBOP_ERR_ARCH = 7,
-    BEBOP_ERR_CUDA = 8
+    BEBOP_ERR_CUDA = 8,
+    BEBOP_ERR_STATIC_SCRATCH = 9
 } bebop_status_t;
 
 typedef enum { BEBOP_F32 = 0, BEBOP_BF16 = 1 } bebop_dtype_t;
@@ -113,6 +114,33 @@ bebop_status_t bebop_tv(
     int N, int V, bebop_dtype_t dt,
     float* tv, float* s_aux, int32_t* row_status,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * bebop_tv without a workspace argument (a convenience of this library; the paper has no
+ * counterpart).  Same computation, same outputs and same errors as bebop_tv, with the per-slice
+ * partials of the sweep kept in a scratch array that is part of the library image
+ * (BEBOP_TV_STATIC_SCRATCH_BYTES = 1 MiB, one copy per device).  The call allocates nothing and
+ * frees nothing.
+ *   - Limit: 24 bytes per (row pair, slice) must fit the array, which holds up to 43,690 of them.
+ *     Rows are cut into fewer slices as N grows (32 for a handful of long rows, 1 beyond a few
+ *     thousand rows), so N up to a few thousand always fits and N > 43,690 never does.  A shape
+ *     that does not fit returns BEBOP_ERR_STATIC_SCRATCH before any launch; use bebop_tv with a
+ *     caller workspace then.
+ *   - Set-up: the first call on each device looks up the device address of the array
+ *     (cudaGetSymbolAddress).  Make that first call before starting a stream capture, not inside
+ *     one; later calls only enqueue kernels and can be captured.
+ *   - The array is shared by every call on the device: two calls that may overlap on the GPU
+ *     (different streams, or graphs replayed concurrently) race on it.  Serialise them, or give
+ *     the overlapping call its own workspace through bebop_tv.
+ *   - Nothing in the array has to start at zero and nothing is kept between calls.
+ */
+#define BEBOP_TV_STATIC_SCRATCH_BYTES (1u << 20)
+bebop_status_t bebop_tv_static(
+    const void* target_logits, int64_t ld_target,
+    const void* draft_logits, int64_t ld_draft,
+    const float* temperature, float temperature_all,
+    int N, int V, bebop_dtype_t dt,
+    float* tv, float* s_aux, int32_t* row_status, void* cuda_stream);
 
 /*
  * Greedy-draft mode (the deterministic limit of target-only sampling, Sec. 2.2):

@@ -7,8 +7,8 @@ calling it without a CUDA device, raises.
 """
 from .binding import (BEBOP_BF16, BEBOP_F32, BebopError, bebop_debug_fallback_offset,
                       bebop_debug_force_general_path, bebop_debug_set_timing_events, bebop_greedy_verify, bebop_status_string,
-                      bebop_tv, bebop_verify, bebop_workspace_bytes, library_path, load_library)
+                      bebop_tv, bebop_tv_static, bebop_verify, bebop_workspace_bytes, library_path, load_library)
 
-__all__ = ["bebop_verify", "bebop_tv", "bebop_greedy_verify", "bebop_workspace_bytes",
+__all__ = ["bebop_verify", "bebop_tv", "bebop_tv_static", "bebop_greedy_verify", "bebop_workspace_bytes",
            "bebop_status_string", "bebop_debug_force_general_path", "bebop_debug_fallback_offset", "bebop_debug_set_timing_events", "BebopError", "BEBOP_F32", "BEBOP_BF16", "library_path",
            "load_library"]

@@ -43,6 +43,8 @@ def load_library():
                                  vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.bebop_tv.restype = i32
     lib.bebop_tv.argtypes = [vp, i64, vp, i64, vp, f32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    lib.bebop_tv_static.restype = i32
+    lib.bebop_tv_static.argtypes = [vp, i64, vp, i64, vp, f32, i32, i32, i32, vp, vp, vp, vp]
     lib.bebop_greedy_verify.restype = i32
     lib.bebop_greedy_verify.argtypes = [vp, i64, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     lib.bebop_debug_force_general_path.restype = None
@@ -189,6 +191,23 @@ def bebop_tv(target_logits, draft_logits, temperature=None, temperature_all=1.0,
     ws, wsb = _workspace(N, 1, V, dt, dev, workspace)
     _check(lib.bebop_tv(tp, ldt, dp, ldd, _ptr(temperature), float(temperature_all), N, V, dt,
                         _ptr(tv), _ptr(s_aux), _ptr(st), _ptr(ws), wsb, _stream()))
+    return dict(tv=tv, s_aux=s_aux, row_status=st)
+
+
+def bebop_tv_static(target_logits, draft_logits, temperature=None, temperature_all=1.0, want_s_aux=True):
+    """bebop_tv with the library's built-in scratch instead of a workspace (no allocation in the call)."""
+    lib = load_library()
+    N, V = target_logits.shape
+    dt = _dt(target_logits)
+    assert draft_logits.dtype == target_logits.dtype and tuple(draft_logits.shape) == (N, V)
+    dev = target_logits.device
+    tp, ldt = _rows(target_logits, 2)
+    dp, ldd = _rows(draft_logits, 2)
+    tv = _new(N, torch.float32, dev)
+    s_aux = _new(N, torch.float32, dev) if want_s_aux else None
+    st = _new(N, torch.int32, dev)
+    _check(lib.bebop_tv_static(tp, ldt, dp, ldd, _ptr(temperature), float(temperature_all), N, V, dt,
+                               _ptr(tv), _ptr(s_aux), _ptr(st), _stream()))
     return dict(tv=tv, s_aux=s_aux, row_status=st)
 
 

@@ -11,6 +11,12 @@ namespace {
 // kernel applies, so that both paths are covered by the parity tests.
 int g_path = 0;   // 0: wave kernel where it applies, otherwise the general kernels
 
+// Built-in scratch of bebop_tv_static: one array per device the module is loaded on.  Nothing in it
+// has to start at zero (every partial is written before it is read).
+static __device__ __align__(256) unsigned char g_tv_scratch[BEBOP_TV_STATIC_SCRATCH_BYTES];
+constexpr int kMaxDevices = 64;
+void* g_tv_scratch_ptr[kMaxDevices] = {nullptr};   // device address of g_tv_scratch, looked up once per device
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Compute capability of the current device, cached per device ordinal.
@@ -141,6 +147,39 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
 
+bebop_status_t bebop_tv_static(const void* target_logits, int64_t ld_target, const void* draft_logits,
+                               int64_t ld_draft, const float* temperature, float temperature_all, int N,
+                               int V, bebop_dtype_t dt, float* tv, float* s_aux, int32_t* row_status,
+                               void* cuda_stream) {
+    bebop_status_t s = check_shape(N, 1, V, dt);
+    if (s != BEBOP_OK) return s;
+    if (!tv) return BEBOP_ERR_NULL;
+    if ((s = check_rows(target_logits, ld_target, V, dt)) != BEBOP_OK) return s;
+    if ((s = check_rows(draft_logits, ld_draft, V, dt)) != BEBOP_OK) return s;
+    if (!temperature && !(temperature_all > 0.f && temperature_all < INFINITY)) return BEBOP_ERR_TEMPERATURE;
+    // the two partial arrays of the TV sweep, packed from the start of the built-in scratch
+    Plan p = make_plan(N, 1, V, (int)dt);
+    const size_t stats_bytes = align256(sizeof(float) * 2 * (size_t)N * 2 * p.nsplit);
+    const size_t zpart_bytes = align256(sizeof(float) * 2 * (size_t)N * p.nsplit);
+    if (stats_bytes + zpart_bytes > BEBOP_TV_STATIC_SCRATCH_BYTES) return BEBOP_ERR_STATIC_SCRATCH;
+    p.off_stats = 0;
+    p.off_zpart = stats_bytes;
+    if ((s = check_arch()) != BEBOP_OK) return s;
+    // set-up, once per device: the device address of the scratch array
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BEBOP_ERR_CUDA;
+    if (!g_tv_scratch_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_tv_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return BEBOP_ERR_CUDA; }
+        g_tv_scratch_ptr[dev] = ptr;
+    }
+    RowArgs a = row_args(target_logits, ld_target, draft_logits, ld_draft, 1, 1, nullptr, temperature,
+                         temperature_all, N, 1, V, dt, p);
+    cudaError_t e = general_tv(a, p, tv, s_aux, row_status, static_cast<char*>(g_tv_scratch_ptr[dev]),
+                               static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
+}
+
 void bebop_debug_force_general_path(int on) { g_path = on; }
 
 void bebop_debug_set_trace(void* p) { wave_set_trace(static_cast<long long*>(p)); }
@@ -163,6 +202,8 @@ const char* bebop_status_string(bebop_status_t status) {
         case BEBOP_ERR_TEMPERATURE: return "temperature_all must be finite and > 0";
         case BEBOP_ERR_ARCH: return "device is not sm_100";
         case BEBOP_ERR_CUDA: return "CUDA launch error";
+        case BEBOP_ERR_STATIC_SCRATCH:
+            return "shape needs more than the built-in scratch of bebop_tv_static: use bebop_tv with a workspace";
     }
     return "unknown status";
 }
