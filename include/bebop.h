@@ -77,8 +77,9 @@ size_t bebop_workspace_bytes(int B, int K, int V, bebop_dtype_t dt);
  *   if all L accepted: draw the bonus token the same way from p_L (target row L)
  *   tv[b,k] = sum_v max(0, p_k - q_k) = d_TV(p_k, q_k) = 1 - E[accept]   (Eq. reject_sample)
  * Rows k >= L are never read; the bonus row is read only when all L are accepted.
- * The draw is evaluated in double precision so that it agrees with an fp64
- * evaluation of the definition except on near-ties.
+ * The draw agrees with an fp64 evaluation of the definition except on near-ties:
+ * an fp32 prefix sum decides the token only where the crossing clears its error
+ * bound on both sides; the remaining sequences are re-drawn in double precision.
  *
  * target_logits [B,K+1,V], draft_logits [B,K,V] : dtype dt
  * draft_tokens  [B,K] int32; draft_len [B] int32 in 0..K, or NULL (= K)
@@ -165,10 +166,14 @@ bebop_status_t bebop_greedy_verify(
  * bebop_debug_set_timing_events(start, stop): two cudaEvent_t handles that the next
  * bebop_verify calls record around the wave kernel, on the caller's stream (NULL,
  * NULL switches it off).
+ * bebop_debug_set_trace(buf): in builds compiled with -DBEBOP_TRACE, a device buffer of
+ * 1024 int64 that the wave kernel fills with per-phase cycle counts (NULL: off); a
+ * no-op in normal builds.
  */
 void bebop_debug_force_general_path(int on);
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
 void bebop_debug_set_timing_events(void* start, void* stop);
+void bebop_debug_set_trace(void* device_buffer);
 
 /* Static, host-side, human-readable name of a status code. */
 const char* bebop_status_string(bebop_status_t status);
