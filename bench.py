@@ -35,10 +35,13 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def ncu_traffic():
-    """DRAM bytes per launch of the wave kernel on the headline workload, from the committed ncu summary."""
+KERNEL_OF_PATH = {0: "k_pipe", 2: "k_wave"}
+
+
+def ncu_traffic(kernel):
+    """DRAM bytes per launch of the dominant kernel on the headline workload, from the committed ncu summary."""
     try:
-        for ln in open(os.path.join(ROOT, "profiles", "k_wave_headline.md")):
+        for ln in open(os.path.join(ROOT, "profiles", kernel + "_headline.md")):
             if ln.startswith("traffic_bytes_per_launch"):
                 return int(ln.split("=")[1].split()[0])
     except Exception:
@@ -46,13 +49,13 @@ def ncu_traffic():
     return None
 
 
-def roofline(alg_bytes, kern_ms, peak, peak_kind, headline):
-    """HBM roofline of the dominant kernel (k_wave): algorithmic bytes of one launch over its
-    CUDA-event duration measured inside the timed region."""
+def roofline(alg_bytes, kern_ms, peak, peak_kind, headline, kernel):
+    """HBM roofline of the dominant kernel: algorithmic bytes of one launch over its CUDA-event
+    duration measured inside the timed region."""
     gbs = alg_bytes / (kern_ms * 1e-3) / 1e9
     return {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-            "traffic": ncu_traffic() if headline else None, "peak_kind": "of " + peak_kind,
-            "kernel": "k_wave", "kernel_ms": kern_ms, "algorithmic_bytes_per_launch": alg_bytes,
+            "traffic": ncu_traffic(kernel) if headline else None, "peak_kind": "of " + peak_kind,
+            "kernel": kernel, "kernel_ms": kern_ms, "algorithmic_bytes_per_launch": alg_bytes,
             "pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS}
 
 
@@ -240,7 +243,7 @@ def run_ours(args):
     kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
     kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = 4 if args.path == 0 else 6      # wave, flag, 2 fp64 re-draw kernels | 6 general kernels
+    launches_per_call = 6 if args.path == 1 else 4      # main kernel, flag, 2 fp64 re-draw kernels | 6 general kernels
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))
@@ -294,7 +297,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3},
             "gpu_launches": steps * launches_per_call,
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,
-            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256 and args.path == 0),
+            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256, KERNEL_OF_PATH.get(args.path, "general kernels")),
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle
@@ -325,7 +328,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: sequences per GPU instead of the workload's 256 (not a bench line)")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
-    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default, 1 general kernels)")
+    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default: pipelined kernel, 1 general kernels, 2 wave kernel)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

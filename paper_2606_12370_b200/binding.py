@@ -91,7 +91,7 @@ def _rows(t: torch.Tensor, ndim: int):
     return C.c_void_p(t.data_ptr()), int(ld)
 
 
-def bebop_debug_force_general_path(on: bool) -> None:
+def bebop_debug_force_general_path(on) -> None:
     load_library().bebop_debug_force_general_path(int(on))
 
 

@@ -52,4 +52,16 @@ cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);
 
+// fp64 re-draw of the sequences a kernel listed (bebop_wave.cu); `w` is the wave workspace laid out by `wp`.
+cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const int* fb_count,
+                          const int* fb_list, char* w, const WavePlan& wp, cudaStream_t stream);
+void wave_flag_launch(const int* wait_failed, int32_t* row_status, int B, cudaStream_t stream);
+
+// Pipelined kernel (bebop_pipe.cu): the wave schedule with a producer warp that stages every task's
+// logits in shared memory by bulk copies while the other warps compute; same contract.
+bool pipe_supported(const RowArgs& a);
+cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

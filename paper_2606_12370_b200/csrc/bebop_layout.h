@@ -7,12 +7,16 @@
 namespace bebop {
 
 // Workspace and schedule parameters of the wave kernel.
-constexpr int kWaveSliceVecs = 2048;   // 16-byte vectors per row slice, at most
+constexpr int kWaveSliceVecs = 2048;   // 16-byte vectors per row slice, at most (wave kernel)
+#ifndef BEBOP_PIPE_SLICE_VECS
+#define BEBOP_PIPE_SLICE_VECS 1536
+#endif
+constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // the same for the pipelined kernel (one stage of its ring)
 struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
     int wave_seqs, nwaves; // sequences per wave, waves
     int lag;               // waves of stats work scheduled between a phase and the phase it depends on
-    size_t off_p1done, off_adone, off_p2done, off_xdone, zero_bytes;
+    size_t off_p1done, off_adone, off_p2done, off_xdone, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
     size_t off_part, off_rstat, off_zpart, off_dpart, off_sinfo, total;
 };
@@ -37,10 +41,10 @@ struct Plan {
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
+static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_cap = kWaveSliceVecs) {
     (void)dt;
     WavePlan w;
-    w.T = (nvec + kWaveSliceVecs - 1) / kWaveSliceVecs; if (w.T < 1) w.T = 1;
+    w.T = (nvec + slice_cap - 1) / slice_cap; if (w.T < 1) w.T = 1;
     w.slice_vecs = (((nvec + w.T - 1) / w.T) + 15) & ~15;   // halves (phase P2) stay 128-byte aligned
     const size_t NR = (size_t)(2 * K + 1);
     const size_t seq_bytes = NR * (size_t)nvec * 16;
@@ -51,10 +55,11 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt) {
     w.nwaves = (B + w.wave_seqs - 1) / w.wave_seqs;
     w.lag = 2;
     size_t o = 256;                                           // ticket, wait flag
-    w.off_p1done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
-    w.off_adone = o;  o += align256(sizeof(int) * (size_t)w.nwaves);
-    w.off_p2done = o; o += align256(sizeof(int) * (size_t)w.nwaves);
+    w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per wave (wave kernel) or per sequence (pipelined kernel)
+    w.off_adone = o;  o += align256(sizeof(int) * (size_t)B);
+    w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
+    w.off_rowcnt = o; o += align256(sizeof(int) * (size_t)B * NR);
     w.zero_bytes = o;
     w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);
     w.off_xmass = o;  o += align256(8 * (size_t)B * 4 * w.T * 8);
@@ -94,7 +99,10 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
-    p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
+    {
+        const size_t w1 = make_wave_plan(B, K, p.nvec, dt).total, w2 = make_wave_plan(B, K, p.nvec, dt, kPipeSliceVecs).total;
+        p.off_wave = o;   o = align256(o + (w1 > w2 ? w1 : w2));
+    }
     p.total = o;
     return p;
 }

@@ -1,0 +1,706 @@
+// Pipelined kernel: the wave schedule (see bebop_wave.cu) with the data movement and the task
+// bookkeeping taken off the compute warps.
+//
+// A CTA is eight consumer warps and one producer warp.  The producer's first lane draws tickets,
+// decodes them (step by step: tickets only grow), checks the wave's completion counter, fetches the
+// few per-task numbers (length, temperature, row normalisers) and, once a stage of the shared-memory
+// ring is free, describes the task there and starts bulk copies (cp.async.bulk, completion counted
+// on the stage's mbarrier) of the slice of logits the task reads: one slice of one row for P1, the
+// same half slice of the target and the draft row for P2, nothing for A and D.  The consumers wait
+// on the stage's barrier, compute from shared memory, and hand the stage back.  A task's partial
+// result is merged by whichever warp finishes last (a shared counter; the merge reads the eight warp
+// partials in warp order, so the result does not depend on who was last), which also publishes it
+// and bumps the wave's completion counter: no CTA-wide barrier sits on the streaming path.
+//
+// Every wait is bounded; a wait that gives up sets the wait flag (status bit 32 of every row).
+// No multicast, no cluster: each CTA copies from this GPU's own memory.
+#define BEBOP_CTA_SYNC() asm volatile("bar.sync 1, 256;" ::: "memory")
+#include "bebop_wave.cuh"
+
+namespace bebop {
+
+namespace {
+
+#ifndef BEBOP_PIPE_STAGES
+#define BEBOP_PIPE_STAGES 3
+#endif
+#ifndef BEBOP_PIPE_CTAS
+#define BEBOP_PIPE_CTAS 3
+#endif
+constexpr int NST = BEBOP_PIPE_STAGES;            // stages of the ring
+constexpr int PIPE_CTAS = BEBOP_PIPE_CTAS;        // CTAs per SM the kernel is built for
+constexpr int PC = WT;                            // consumer threads (8 warps); thread PC is the producer
+constexpr int PT = PC + 64;                       // + producer warp + publisher warp
+constexpr int PSLICE = kPipeSliceVecs;            // vectors per stage
+constexpr int STAGE_BYTES = PSLICE * 16;
+constexpr int kPend = 4;                          // runs a producer may set aside
+#ifndef BEBOP_PIPE_BATCH
+#define BEBOP_PIPE_BATCH 2
+#endif
+constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time
+constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
+
+struct __align__(16) TaskDesc {
+    int phase;        // 0 P1, 1 A, 2 P2, 3 D, -1: no more tasks
+    int wave, b, r;   // r: row (P1) or draft position (P2)
+    int s, v0, nv;    // slice, its first vector, its vectors
+    int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from
+    float tau;
+    RowScale P, Q;
+#ifdef BEBOP_TRACE
+    long long t_issue;
+#endif
+};
+
+struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of one (phase, wave) block from offset off
+
+struct PipeShared {
+    WaveShared W;                               // scratch of phases A and D
+    TaskDesc desc[NST];
+    unsigned long long full[NST], empty[NST];   // mbarriers: data and description there / stage free again
+    unsigned long long pdone[NST];              // mbarrier: the eight warp partials of the stage's task are there
+    float wf[NST][2][WW];                       // per-warp partials of the task in the stage
+    double wd[NST][WW];
+    int wi[NST][WW];
+    Run pend[kPend];                            // producer: runs set aside
+#ifdef BEBOP_TRACE
+    long long t_empty[NST];
+#endif
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* b, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(unsigned long long* b, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity) {
+    const uint32_t addr = smem_u32(b);
+    for (uint32_t i = 0; i < kBarSpin; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// contiguous copy global -> shared of this CTA; 16-byte aligned on both sides, size a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ void release_add(int* p) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" :: "l"(p) : "memory");
+}
+
+#ifdef BEBOP_TRACE
+// per wave timeline (ns): [64 + 8*w + i]: 0 first P1 ticket, 1 last row merged, 2 last accept done, 3 first P2 ticket seen,
+// 4 first P2 task published, 5 last P2 partial done, 6 first D ticket seen, 7 last D done
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ void tl_min(const WaveArgs& a, int w, int i) { if (a.trace) atomicMin(reinterpret_cast<unsigned long long*>(a.trace) + 64 + 8 * w + i, (unsigned long long)gtime()); }
+__device__ __forceinline__ void tl_max(const WaveArgs& a, int w, int i) { if (a.trace) atomicMax(reinterpret_cast<unsigned long long*>(a.trace) + 64 + 8 * w + i, (unsigned long long)gtime()); }
+#define TL_MIN(w, i) tl_min(a, w, i)
+#define TL_MAX(w, i) tl_max(a, w, i)
+#else
+#define TL_MIN(w, i) do { } while (0)
+#define TL_MAX(w, i) do { } while (0)
+#endif
+
+// ------------------------------------------------------------------ producer
+// One thread.  Tickets are claimed kBatch at a time; consecutive tickets of one (phase, wave) block are
+// consecutive slices of a row, then the next row, then the next sequence, so a batch decodes once and
+// then steps, and the per-row numbers (length, temperature, normalisers, row addresses) are fetched
+// once per row.  Returns when the stop description has been handed to the consumers.
+template <int DT>
+__device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsigned char* data) {
+    const RowArgs& R = a.r;
+    const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
+    const int B = R.B;
+    const int c0 = NR * T, c2 = (K + 1) * T2;
+    const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
+    // Ticket order: all of P1 (sequences ascending), then all of P2 and then all of D with the sequences
+    // DESCENDING: the last sequences P1 streamed are the ones still in L2 when P2 begins.  Every logit comes
+    // from DRAM once per sweep except that tail.  Phase A has no tickets: it runs in the warp that
+    // completes a sequence's last softmax partial, long before P2 asks for it.
+    const int n1 = B * c0, n2 = B * c2;
+    // the run of block-consecutive tasks that starts at ticket t and has at most `want` tasks
+    auto decode = [&](int t, int want) {
+        Run r;
+        r.wv = 0;
+        int room;
+        if (t < n1) { r.ph = 0; r.off = t; room = n1 - t; }
+        else if (t < n1 + n2) { r.ph = 2; r.off = t - n1; room = n1 + n2 - t; }
+        else { r.ph = 3; r.off = t - n1 - n2; room = a.ntickets - t; }
+        r.cnt = min(want, room);
+        return r;
+    };
+    // Is sequence b ready for the phase?  P2 needs its accept scan, D all of its P2 partials.  A run that is
+    // not ready is set aside (up to kPend of them) while later tickets go ahead; the oldest one is looked at
+    // again before every new run and waited for only when the shelf is full or no tickets are left.
+    auto ready = [&](int ph, int b, bool wait) {
+        if (ph == 2) return wait ? spin_ge(&a.adone[b], 1) : ld_acquire(&a.adone[b]) >= 1;
+        if (ph == 3) return wait ? spin_ge(&a.p2done[b], c2) : ld_acquire(&a.p2done[b]) >= c2;
+        return true;
+    };
+    // first sequence of a run (runs are cut at sequence boundaries for P2 and D, see below)
+    auto run_seq = [&](const Run& r) { return r.ph == 0 ? r.off / c0 : (r.ph == 2 ? B - 1 - r.off / c2 : B - 1 - r.off); };
+#ifdef BEBOP_TRACE
+    long long qprev_ = clock64();
+#endif
+    int npend = 0;
+    bool exhausted = false;
+    int bt = 0, bleft = 0;                         // tickets of the claimed batch not yet turned into runs
+    int next = atomicAdd(a.ticket, kBatch);
+    int it = 0;
+    for (;;) {
+        // ---- next run
+        Run run;
+        if (npend > 0 && (ready(S.pend[0].ph, run_seq(S.pend[0]), false) || npend == kPend || (exhausted && bleft == 0))) {
+            run = S.pend[0];
+            if (!ready(run.ph, run_seq(run), true)) atomicExch(a.wait_failed, 1);
+            --npend;
+            for (int i = 0; i < npend; ++i) S.pend[i] = S.pend[i + 1];
+        } else {
+            if (bleft == 0 && !exhausted) {
+                bt = next; bleft = min(kBatch, a.ntickets - bt);
+                if (bleft <= 0) { bleft = 0; exhausted = true; }
+                else next = atomicAdd(a.ticket, kBatch);
+            }
+            if (bleft == 0) {
+                if (npend > 0) continue;
+                const int stage = it % NST;
+                if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
+                S.desc[stage].phase = -1;
+                mbar_arrive(&S.full[stage]);
+                return;
+            }
+            run = decode(bt, bleft);
+            // a P2 or D run stays within one sequence, so that one readiness check covers it
+            if (run.ph == 2) run.cnt = min(run.cnt, c2 - run.off % c2); else if (run.ph == 3) run.cnt = 1;
+            bt += run.cnt; bleft -= run.cnt;
+            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; continue; }
+        }
+        // ---- the tasks of the run
+        const int ph = run.ph, wv = 0;
+        const int per_row = ph == 0 ? T : (ph == 2 ? T2 : 1), rows = ph == 0 ? NR : (ph == 2 ? K + 1 : 1);
+        int s = run.off % per_row, r = (run.off / per_row) % rows, bb = run.off / (per_row * rows);
+        int left = run.cnt;
+        while (left > 0) {
+            const int b = ph == 0 ? bb : B - 1 - bb;
+            // the row's numbers
+            TaskDesc d;
+            d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f;
+            d.P = no_row(); d.Q = no_row();
+            const char* row0 = nullptr; const char* row1 = nullptr;
+            bool skip = false;
+            int* done = nullptr;
+            if (ph == 0) {
+                const int L = len_of(R, b);
+                const bool is_target = r <= K;
+                const int k = is_target ? r : r - (K + 1);
+                d.tau = tau_of(R, b);
+                skip = is_target ? k > L : k >= L;
+                row0 = row_ptr(R, b, r);
+            } else if (ph == 2) {
+                const int k = r, L = len_of(R, b);
+                d.tau = tau_of(R, b);
+                done = &a.p2done[b];
+                skip = k > L;
+                if (!skip) {
+                    const SeqInfo si = ld_cg(a.sinfo + b);
+                    const RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
+                    const RowStat sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + min(k, K - 1));
+                    const bool pair = k < L;
+                    skip = si.n < 0 || (!pair && si.draw_row != L);
+                    if (!skip) {
+                        d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
+                        d.P = row_scale(sp);
+                        if (pair) d.Q = row_scale(sq);
+                        row0 = row_ptr(R, b, k);
+                        if (pair) row1 = row_ptr(R, b, K + 1 + k);
+                    }
+                }
+            }
+            const int n_row = min(left, per_row - s);         // tasks of this run in this row
+            if (skip) {
+                if (done) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" :: "l"(done), "r"(n_row) : "memory");
+            } else {
+                const int sv = ph == 0 ? sv1 : sv2;
+                for (int i = 0; i < n_row; ++i) {
+                    const int stage = it % NST;
+                    d.s = s + i; d.v0 = d.s * sv; d.nv = max(min(sv, R.nvec - d.v0), 0);
+#ifdef BEBOP_TRACE
+                    const long long q0_ = clock64();
+#endif
+                    if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
+#ifdef BEBOP_TRACE
+                    const long long q1_ = clock64();
+                    d.t_issue = q1_;
+                    if (a.trace && a.trace[4095] != 0) {
+                        unsigned long long* tq = reinterpret_cast<unsigned long long*>(a.trace) + 32 + ph * 8;
+                        atomicAdd(tq + 0, (unsigned long long)(q0_ - qprev_)); atomicAdd(tq + 1, (unsigned long long)(q1_ - q0_)); atomicAdd(tq + 2, 1ull);
+                        if (it >= NST) atomicAdd(tq + 3, (unsigned long long)(q1_ - S.t_empty[stage]));
+                    }
+                    qprev_ = q1_;
+                    if (a.trace && blockIdx.x == 5 && it < 100) { a.trace[2048 + it * 20] = q1_; a.trace[2048 + it * 20 + 17] = ph; }
+#endif
+                    S.desc[stage] = d;
+                    const uint32_t bytes = (uint32_t)d.nv * 16u;
+                    if (row0 && bytes) {
+                        mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
+                        bulk_load(data + (size_t)stage * STAGE_BYTES, row0 + (int64_t)d.v0 * 16, bytes, &S.full[stage]);
+                        if (row1) bulk_load(data + (size_t)stage * STAGE_BYTES + STAGE_BYTES / 2, row1 + (int64_t)d.v0 * 16, bytes, &S.full[stage]);
+                    } else {
+                        mbar_arrive(&S.full[stage]);
+                    }
+                    ++it;
+                }
+            }
+            left -= n_row;
+            s = 0;
+            if (++r == rows) { r = 0; ++bb; }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ phase A without tickets
+// The warp that delivers the last softmax partial of a ROW merges that row's partials (exactly:
+// integer exponents, fp64 sums in a fixed tree) and leaves the row's normaliser; the warp that merges
+// the last row of a SEQUENCE runs the accept scan at once and writes accept_len, the accepted tokens,
+// p(x), q(x), the status and the stop position.  No ticket, no CTA barrier, and the work is done
+// long before phase P2 of the wave is handed out.
+__device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) {
+    const int lane = threadIdx.x & 31;
+    const int NR = 2 * a.r.K + 1, T = a.T;
+    const P1Part* pp = a.part + ((int64_t)b * NR + r) * T;
+    // lanes take slices in order; exponent first, then the scaled sum in a fixed tree
+    int e_l = E_EMPTY; double s_l = 0.0; int f_l = 0;
+    P1Part mine[2];
+    int cnt = 0;
+    for (int s = lane; s < T && cnt < 2; s += 32) {
+        mine[cnt] = ld_cg(pp + s); e_l = max(e_l, mine[cnt].e);
+        if (mine[cnt].m != mine[cnt].m) f_l = 1;
+        cnt++;
+    }
+    const int Em = redux_max(e_l);
+    for (int i = 0; i < cnt; ++i) if (mine[i].e > E_EMPTY) s_l += mine[i].s * pow2d(max(mine[i].e - Em, -1000));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { s_l += shfl_xor_d(s_l, o); f_l |= __shfl_xor_sync(0xffffffffu, f_l, o); }
+    if (lane == 0) {
+        int st = 0;
+        if (f_l || !(s_l == s_l)) st = ST_NONFINITE; else if (Em == E_EMPTY) st = ST_EMPTY;
+        RowStat rs; rs.inv_s = (!st && s_l > 0.0) ? 1.0 / s_l : 0.0; rs.ef = (float)Em; rs.e = Em; rs.pad[0] = st; rs.pad[1] = 0;
+        a.rstat[(int64_t)b * NR + r] = rs;
+    }
+}
+
+template <int DT>
+__device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
+    const RowArgs& R = a.r;
+    const int lane = threadIdx.x & 31;
+    const int K = R.K, V = R.V, L = len_of(R, b), NR = 2 * K + 1;
+    const float tau = tau_of(R, b);
+    const bool ok = tau_ok(tau);
+    const TempScale ts = temp_scale(tau);
+    // lane k owns draft position k (K <= 32): everything it needs is requested before anything is used
+    const bool active = lane < L;
+    const int tk = active ? a.draft_tokens[(int64_t)b * K + lane] : 0;
+    const float u = active ? a.u_accept[(int64_t)b * K + lane] : 0.f;
+    RowStat sp, sq, sb;
+    sp.inv_s = 0.0; sp.ef = 0.f; sp.e = E_EMPTY; sp.pad[0] = 0; sp.pad[1] = 0;
+    sq = sp;
+    if (active) { sp = ld_cg(a.rstat + (int64_t)b * NR + lane); sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + lane); }
+    sb = ld_cg(a.rstat + (int64_t)b * NR + L);                         // bonus row (row L <= K: always merged)
+    int seq_st = ok ? 0 : ST_BAD_TEMP;
+    const bool tok_ok = tk >= 0 && tk < V;
+    float zpx = 0.f, zqx = 0.f;
+    if (active && tok_ok) { zpx = load_one<DT>(row_ptr(R, b, lane), tk); zqx = load_one<DT>(row_ptr(R, b, K + 1 + lane), tk); }
+    if (!seq_st && __ballot_sync(0xffffffffu, active && !tok_ok)) seq_st = ST_BAD_TOKEN;
+    // the first bad row pair decides the status; rows after it do not count
+    const int rs = active ? (sp.pad[0] | sq.pad[0]) : 0;
+    const unsigned badrows = __ballot_sync(0xffffffffu, rs != 0);
+    const int first_bad = badrows ? __ffs(badrows) - 1 : 32;
+    const int rs_first = __shfl_sync(0xffffffffu, rs, first_bad & 31);
+    if (!seq_st && badrows) seq_st = rs_first;
+    double px = 0.0, qx = 0.0;
+    bool acc = false;
+    if (active && !(seq_st & ST_FATAL) && lane < first_bad) {
+        const double cd = (double)ts.hi;
+        px = exp2((double)zpx * cd - (double)sp.e) * sp.inv_s;
+        qx = exp2((double)zqx * cd - (double)sq.e) * sq.inv_s;
+        acc = (double)u * qx < px;
+    }
+    const unsigned rej = __ballot_sync(0xffffffffu, active && !acc);
+    const int n = rej ? __ffs(rej) - 1 : L;
+    if (!(seq_st & ST_FATAL) && n == L && sb.pad[0]) seq_st |= sb.pad[0];   // bonus row, counted only now
+    const bool fatal = (seq_st & ST_FATAL) != 0;
+    const int nn = fatal ? 0 : n;
+    // outputs: lane q writes position q (position nn is filled by the draw)
+    for (int q = lane; q <= K; q += 32)
+        if (fatal || q != nn) a.o.out_tokens[(int64_t)b * (K + 1) + q] = q < nn ? tk : -1;   // q < nn <= 32: q == lane
+    if (lane < K) {
+        const bool zero = fatal || lane >= L;
+        if (a.o.p_draft) a.o.p_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)px;
+        if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)qx;
+        if (zero && a.o.tv) a.o.tv[(int64_t)b * K + lane] = 0.f;
+    }
+    if (lane == 0) {
+        a.o.accept_len[b] = nn;
+        if (a.o.row_status) a.o.row_status[b] = seq_st;
+        a.stop[b] = fatal ? -1 : nn;
+        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = 0; si.pad = 0;
+        a.sinfo[b] = si;
+        __threadfence();
+        release_add(&a.adone[b]);
+    }
+}
+
+// ------------------------------------------------------------------ consumers
+// Each consumer warp leaves its partial of a task in shared memory and signals the stage's `pdone` barrier;
+// the publisher warp merges the eight partials in warp order and publishes the result, off the consumers'
+// path.
+__device__ __forceinline__ int add_acq_rel(int* p, int v) {
+    int old;
+    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
+// P1: softmax partial (E, S) of one slice of one row, from shared memory.
+template <int DT>
+__device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+                                        int stage, int it) {
+    constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
+    const RowArgs& R = a.r;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const TempScale ts = temp_scale(d.tau);
+    const int nv = d.nv;
+    uint4 raw[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        const int v = tid + u * PC;
+        raw[u] = neg_inf_vec<DT>();
+        if (v < nv) raw[u] = lds16(data + (size_t)v * 16);
+    }
+    if ((d.v0 + nv) * VEC > R.V) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int gbase = (d.v0 + tid + u * PC) * VEC;
+            if (tid + u * PC < nv && gbase + VEC > R.V) mask_tail<DT>(raw[u], R.V - gbase);
+        }
+    }
+    float m = vec_max<DT>(raw[0]);
+#pragma unroll
+    for (int u = 1; u < NV; ++u) m = max_nan(m, vec_max<DT>(raw[u]));
+    const bool bad = m != m || m == INFINITY;
+    int E = E_EMPTY;
+    float Ef = 0.f;
+    if (!bad && m != -INFINITY) E = ref_exponent(m, ts, &Ef);
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    if (E > E_EMPTY) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            float f[VEC];
+            unpack<DT>(raw[u], f);
+#pragma unroll
+            for (int i = 0; i < VEC; i += 4) {
+                s0 += exp2_scaled(f[i], ts, Ef);
+                s1 += exp2_scaled(f[i + 1], ts, Ef);
+                s2 += exp2_scaled(f[i + 2], ts, Ef);
+                s3 += exp2_scaled(f[i + 3], ts, Ef);
+            }
+        }
+    }
+    // thread -> warp, exact power-of-two rescaling, sums in a fixed order
+    float st = (s0 + s1) + (s2 + s3);
+    const int Ew = redux_max(E);
+    st = E > E_EMPTY ? st * pow2f(max(E - Ew, -126)) : 0.f;
+    st = warp_sum(st);
+    const unsigned anybad = __ballot_sync(0xffffffffu, bad);
+    float mw = ord2f(redux_max(f2ord(bad ? -INFINITY : m)));
+    if (anybad) mw = __int_as_float(0x7fc00000);
+    if (lane == 0) { S.wf[stage][0][warp] = st; S.wi[stage][warp] = Ew; S.wf[stage][1][warp] = mw; }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&S.pdone[stage]);
+}
+
+// P2: TV partial of one half slice of a row pair; on the pair (or bonus row) a token is drawn from,
+// also the mass in double and the sum of squares.  Target row in the first half of the stage, draft
+// row in the second.
+template <int DT>
+__device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+                                        int stage, int it) {
+    constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / (2 * PC);
+    const RowArgs& R = a.r;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool pair = (d.flags & 1) != 0, draw = (d.flags & 2) != 0;
+    const int nv = d.nv;
+    const unsigned char* qdata = data + STAGE_BYTES / 2;
+    uint4 rp[NV], rq[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        const int v = tid + u * PC;
+        rp[u] = neg_inf_vec<DT>(); rq[u] = neg_inf_vec<DT>();
+        if (v < nv) { rp[u] = lds16(data + (size_t)v * 16); if (pair) rq[u] = lds16(qdata + (size_t)v * 16); }
+    }
+    const TempScale c = temp_scale(d.tau);
+    const RowScale SP = d.P, SQ = d.Q;
+    if ((d.v0 + nv) * VEC > R.V) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int gbase = (d.v0 + tid + u * PC) * VEC;
+            if (tid + u * PC < nv && gbase + VEC > R.V) { mask_tail<DT>(rp[u], R.V - gbase); mask_tail<DT>(rq[u], R.V - gbase); }
+        }
+    }
+    float z0 = 0.f, z1 = 0.f, sqs = 0.f;
+    double zd = 0.0;
+    if (!draw) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            if (tid + u * PC < nv) {
+                float r[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                residual_vec<DT, false>(rp[u], rq[u], pair, c, SP, SQ, r, nullptr);
+                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                if (u & 1) z1 += vs; else z0 += vs;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            if (tid + u * PC < nv) {
+                float r[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                residual_vec<DT, true>(rp[u], rq[u], pair, c, SP, SQ, r, &sqs);
+                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                z0 += vs;
+                zd += (double)vs;
+            }
+        }
+    }
+    const float z = warp_sum(z0 + z1);
+    if (draw) { zd = warp_sum(zd); sqs = warp_sum(sqs); }
+    if (lane == 0) { S.wf[stage][0][warp] = z; S.wd[stage][warp] = zd; S.wf[stage][1][warp] = sqs; }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&S.pdone[stage]);
+}
+
+// ------------------------------------------------------------------ publisher
+// One warp.  For every streaming task: wait for the eight warp partials, take them into registers,
+// hand the stage back, then merge (warp order, so the result does not depend on timing) and publish:
+// P1 -- the slice's (E, S) partial and the row's counter, whose last increment starts the merge of the
+// row, whose last merged row starts the accept scan of the sequence; P2 -- the TV part (and the
+// draw-row mass) and the sequence's counter.
+template <int DT>
+__device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
+    const RowArgs& R = a.r;
+    const int lane = threadIdx.x & 31;
+    const int K = R.K, T2 = 2 * a.T;
+    for (int it = 0;; ++it) {
+        const int stage = it % NST;
+        const uint32_t par = (uint32_t)(it / NST) & 1u;
+        if (!mbar_wait(&S.full[stage], par)) { if (lane == 0) atomicExch(a.wait_failed, 1); return; }
+        const int phase = S.desc[stage].phase;
+        if (phase < 0) return;
+        if (phase != 0 && phase != 2) {                       // D: nothing to publish
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.empty[stage]);
+            continue;
+        }
+        if (!mbar_wait(&S.pdone[stage], par)) { if (lane == 0) atomicExch(a.wait_failed, 1); return; }
+        const int b = S.desc[stage].b, r = S.desc[stage].r, sl = S.desc[stage].s, flags = S.desc[stage].flags;
+        const int w = lane & (WW - 1);
+        const float f0 = S.wf[stage][0][w], f1 = S.wf[stage][1][w];
+        const double dd = S.wd[stage][w];
+        const int ii = S.wi[stage][w];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&S.empty[stage]);
+        if (phase == 0) {
+            // lanes 0..7 hold the warps' (sum, exponent, max); merge in warp order
+            const int Ec = max(max(max(__shfl_sync(0xffffffffu, ii, 0), __shfl_sync(0xffffffffu, ii, 1)),
+                                   max(__shfl_sync(0xffffffffu, ii, 2), __shfl_sync(0xffffffffu, ii, 3))),
+                               max(max(__shfl_sync(0xffffffffu, ii, 4), __shfl_sync(0xffffffffu, ii, 5)),
+                                   max(__shfl_sync(0xffffffffu, ii, 6), __shfl_sync(0xffffffffu, ii, 7))));
+            const double mine = ii > E_EMPTY ? (double)(f0 * pow2f(max(ii - Ec, -126))) : 0.0;
+            double sum = 0.0; float mc = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < WW; ++k) { sum += __shfl_sync(0xffffffffu, mine, k); mc = max_nan(mc, __shfl_sync(0xffffffffu, f1, k)); }
+            int run_a = 0;
+            if (lane == 0) {
+                P1Part p; p.s = (mc != mc) ? 0.0 : sum; p.e = Ec; p.m = mc;
+                a.part[((int64_t)b * (2 * K + 1) + r) * a.T + sl] = p;
+                // the last softmax partial of a row starts the merge of that row (release: the partial above;
+                // acquire: the partials of the other slices)
+                run_a = add_acq_rel(&a.rowcnt[(int64_t)b * (2 * K + 1) + r], 1) == a.T - 1;
+            }
+            if (__shfl_sync(0xffffffffu, run_a, 0)) {
+                merge_row_warp(a, b, r);
+                // the last merged row of the sequence (2L+1 rows are in use) starts the accept scan
+                int last_row = 0;
+                if (lane == 0) last_row = add_acq_rel(&a.p1done[b], 1) == 2 * len_of(R, b);
+                if (__shfl_sync(0xffffffffu, last_row, 0)) accept_warp<DT>(a, b);
+            }
+        } else {
+            float zz = 0.f, sq = 0.f; double tot = 0.0;
+#pragma unroll
+            for (int k = 0; k < WW; ++k) {
+                zz += __shfl_sync(0xffffffffu, f0, k); sq += __shfl_sync(0xffffffffu, f1, k); tot += __shfl_sync(0xffffffffu, dd, k);
+            }
+            if (lane == 0) {
+                if (flags & 1) a.zpart[((int64_t)b * K + r) * T2 + sl] = zz;
+                if (flags & 2) { DPart dp; dp.tot = tot; dp.sq = sq; dp.pad = 0; a.dpart[(int64_t)b * T2 + sl] = dp; }
+                release_add(&a.p2done[b]);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+template <int DT>
+__global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ WaveArgs a) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* data = smem;
+    PipeShared& S = *reinterpret_cast<PipeShared*>(smem + (size_t)NST * STAGE_BYTES);
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        for (int i = 0; i < NST; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], WW + 1); mbar_init(&S.pdone[i], WW); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid >= PC) {
+        if (tid == PC) producer<DT>(a, S, data);
+        else if (tid >= PC + 32) publisher<DT>(a, S);
+        return;
+    }
+    const int lane = tid & 31;
+    for (int it = 0;; ++it) {
+        const int stage = it % NST;
+        const uint32_t par = (uint32_t)(it / NST) & 1u;
+#ifdef BEBOP_TRACE
+        const long long c0_ = clock64();
+#endif
+        if (!mbar_wait(&S.full[stage], par)) { if (tid == 0) atomicExch(a.wait_failed, 1); break; }
+        const TaskDesc d = S.desc[stage];
+        if (d.phase < 0) break;
+#ifdef BEBOP_TRACE
+        const long long c1_ = clock64();
+#endif
+        const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
+        if (d.phase == 0) pipe_p1<DT>(a, S, d, sd, stage, it);
+        else if (d.phase == 2) pipe_p2<DT>(a, S, d, sd, stage, it);
+        else {
+            if (tid == 0) S.W.vsum = reinterpret_cast<float*>(data + (size_t)stage * STAGE_BYTES);   // a D task's stage holds no logits
+            phase_d<DT>(a, S.W, d.b);
+            BEBOP_CTA_SYNC();
+
+        }
+        __syncwarp();
+#ifdef BEBOP_TRACE
+        if (lane == 0) S.t_empty[stage] = clock64();
+#endif
+        if (lane == 0) mbar_arrive(&S.empty[stage]);
+#ifdef BEBOP_TRACE
+        if (a.trace && lane == 0 && blockIdx.x == 5 && it < 100) { a.trace[2048 + it * 20 + 1 + (tid >> 5)] = c1_; a.trace[2048 + it * 20 + 9 + (tid >> 5)] = clock64(); }
+        if (a.trace && lane == 0 && a.trace[4095] != 0) {       // per phase and warp-task: cycles waiting for the stage, cycles of the task, count
+            unsigned long long* tq = reinterpret_cast<unsigned long long*>(a.trace) + d.phase * 8;
+            atomicAdd(tq + 0, (unsigned long long)(c1_ - c0_)); atomicAdd(tq + 1, (unsigned long long)(clock64() - c1_));
+            atomicAdd(tq + 2, 1ull);
+            atomicAdd(tq + 3, (unsigned long long)(c1_ - d.t_issue));
+        }
+#endif
+    }
+}
+
+// -----------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kPipeSmem = (size_t)NST * STAGE_BYTES + sizeof(PipeShared);
+
+template <int DT>
+int pipe_grid() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
+    if (cudaFuncSetAttribute(k_pipe<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    int per_sm = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pipe<DT>, PT, kPipeSmem) != cudaSuccess) per_sm = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaGetLastError();
+    const int n = per_sm * sms;
+    if (dev >= 0 && dev < 64) cached[dev] = n;
+    return n;
+}
+
+}  // namespace
+
+extern long long* g_wave_trace;
+extern cudaEvent_t g_ev_start, g_ev_stop;
+
+bool pipe_supported(const RowArgs& a) {
+    const int T = (a.nvec + PSLICE - 1) / PSLICE;
+    return T >= 1 && T <= MAX_SLICES && a.K <= BEBOP_MAX_K_INT;
+}
+
+cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched) {
+    *launched = false;
+    const int grid_max = a.dt == 0 ? pipe_grid<0>() : pipe_grid<1>();
+    if (grid_max < 1) return cudaSuccess;
+    const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
+    WaveArgs wa;
+    wa.r = a; wa.draft_tokens = draft_tokens; wa.u_accept = u_accept; wa.u_final = u_final; wa.o = o;
+    wa.stop = reinterpret_cast<int*>(ws + p.off_stop);
+    wa.fb_count = reinterpret_cast<int*>(ws + p.off_fb);
+    wa.fb_list = wa.fb_count + 16;
+    char* w = ws + p.off_wave;
+    wa.ticket = reinterpret_cast<int*>(w);
+    wa.wait_failed = wa.ticket + 1;
+    wa.p1done = reinterpret_cast<int*>(w + wp.off_p1done);
+    wa.adone = reinterpret_cast<int*>(w + wp.off_adone);
+    wa.p2done = reinterpret_cast<int*>(w + wp.off_p2done);
+    wa.rowcnt = reinterpret_cast<int*>(w + wp.off_rowcnt);
+    wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
+    wa.rstat = reinterpret_cast<RowStat*>(w + wp.off_rstat);
+    wa.zpart = reinterpret_cast<float*>(w + wp.off_zpart);
+    wa.dpart = reinterpret_cast<DPart*>(w + wp.off_dpart);
+    wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
+    wa.trace = g_wave_trace;
+    wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;
+    {
+        const long long NR = 2 * a.K + 1;
+        const long long total = (long long)a.B * (NR * wp.T + (long long)(a.K + 1) * 2 * wp.T + 1);
+        if (total > 0x7fff0000LL) return cudaSuccess;
+        wa.ntickets = (int)total;
+        wa.lag = wp.lag;
+    }
+    cudaError_t e = cudaMemsetAsync(w, 0, wp.zero_bytes, stream);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(wa.fb_count, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return e;
+    const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
+    if (g_ev_start) cudaEventRecord(g_ev_start, stream);
+    if (a.dt == 0) k_pipe<0><<<grid, PT, kPipeSmem, stream>>>(wa);
+    else k_pipe<1><<<grid, PT, kPipeSmem, stream>>>(wa);
+    e = cudaGetLastError();
+    if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
+    if (e != cudaSuccess) return e;
+    wave_flag_launch(wa.wait_failed, o.row_status, a.B, stream);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    *launched = true;
+    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, w, wp, stream);
+}
+
+}  // namespace bebop

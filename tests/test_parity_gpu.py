@@ -15,13 +15,16 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.fixture(autouse=True, params=["wave", "general"])
+PATHS = {"pipe": 0, "general": 1, "wave": 2}
+
+
+@pytest.fixture(autouse=True, params=["pipe", "wave", "general"])
 def kernel_path(request):
-    """Every test runs twice: through the fused cluster kernel where the shape admits it,
-    and through the general split-row kernels."""
-    P.bebop_debug_force_general_path(request.param == "general")
+    """Every test runs three times: through the pipelined kernel and the wave kernel where the shape
+    admits them, and through the general split-row kernels."""
+    P.bebop_debug_force_general_path(PATHS[request.param])
     yield request.param
-    P.bebop_debug_force_general_path(False)
+    P.bebop_debug_force_general_path(0)
 
 
 def run_verify(x, **kw):
