@@ -148,7 +148,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         return true;
     };
     // first sequence of a run (runs are cut at sequence boundaries for P2 and D, see below)
-    auto run_seq = [&](const Run& r) { return r.ph == 0 ? r.off / c0 : (r.ph == 2 ? B - 1 - r.off / c2 : B - 1 - r.off); };
+    auto run_seq = [&](const Run& r) { return r.ph == 0 ? r.off / c0 : (r.ph == 2 ? r.off / c2 : r.off); };
 #ifdef BEBOP_TRACE
     long long qprev_ = clock64();
 #endif
@@ -191,7 +191,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         int s = run.off % per_row, r = (run.off / per_row) % rows, bb = run.off / (per_row * rows);
         int left = run.cnt;
         while (left > 0) {
-            const int b = ph == 0 ? bb : B - 1 - bb;
+            const int b = bb;
             // the row's numbers
             TaskDesc d;
             d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f;
