@@ -502,6 +502,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, T2 = 2 * a.T;
+    uint32_t pd_par = 0;                                      // per stage: parity of the next `pdone` phase
     for (int it = 0;; ++it) {
         const int stage = it % NST;
         const uint32_t par = (uint32_t)(it / NST) & 1u;
@@ -513,7 +514,10 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
             if (lane == 0) mbar_arrive(&S.empty[stage]);
             continue;
         }
-        if (!mbar_wait(&S.pdone[stage], par)) { if (lane == 0) atomicExch(a.wait_failed, 1); return; }
+        // `pdone` only advances on streaming tasks (a D task leaves no partials), so its phase is tracked per
+        // stage rather than derived from the task number
+        if (!mbar_wait(&S.pdone[stage], (pd_par >> stage) & 1u)) { if (lane == 0) atomicExch(a.wait_failed, 1); return; }
+        pd_par ^= 1u << stage;
         const int b = S.desc[stage].b, r = S.desc[stage].r, sl = S.desc[stage].s, flags = S.desc[stage].flags;
         const int w = lane & (WW - 1);
         const float f0 = S.wf[stage][0][w], f1 = S.wf[stage][1][w];
