@@ -35,7 +35,7 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-KERNEL_OF_PATH = {0: "k_pipe", 2: "k_wave"}
+KERNEL_OF_PATH = {0: "k_pipe"}
 
 
 def ncu_traffic(kernel):
@@ -219,7 +219,7 @@ def run_ours(args):
         step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # events around the dominant kernel (the wave kernel) inside the timed region: the library records
+    # events around the dominant kernel (k_pipe) inside the timed region: the library records
     # them on the launching stream; at most 256 steps carry a pair
     stride = max(1, steps // 256)
     pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -328,7 +328,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: sequences per GPU instead of the workload's 256 (not a bench line)")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
-    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default: pipelined kernel, 1 general kernels, 2 wave kernel)")
+    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default: pipelined kernel, 1 general kernels)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

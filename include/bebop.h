@@ -159,15 +159,15 @@ bebop_status_t bebop_greedy_verify(
 /*
  * Test and measurement hooks (no counterpart in the paper).
  * bebop_debug_force_general_path(1) makes bebop_verify use the split-row general
- * kernels even for shapes the wave kernel takes (process-wide switch; 0 restores).
+ * kernels even for shapes the pipelined kernel takes (process-wide switch; 0 restores).
  * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
  * shape, of an int32 that after a bebop_verify call holds the number of sequences
  * whose draw was re-done by the fp64 kernels.
  * bebop_debug_set_timing_events(start, stop): two cudaEvent_t handles that the next
- * bebop_verify calls record around the wave kernel, on the caller's stream (NULL,
+ * bebop_verify calls record around the pipelined kernel, on the caller's stream (NULL,
  * NULL switches it off).
  * bebop_debug_set_trace(buf): in builds compiled with -DBEBOP_TRACE, a device buffer of
- * 1024 int64 that the wave kernel fills with per-phase cycle counts (NULL: off); a
+ * int64 that the pipelined kernel fills with cycle counts (NULL: off); a
  * no-op in normal builds.
  */
 void bebop_debug_force_general_path(int on);

@@ -96,7 +96,7 @@ def bebop_debug_force_general_path(on) -> None:
 
 
 def bebop_debug_set_timing_events(start, stop) -> None:
-    """torch.cuda.Event pair (enable_timing=True, already recorded once) bracketing the wave kernel; None, None = off."""
+    """torch.cuda.Event pair (enable_timing=True, already recorded once) bracketing the main (pipelined) kernel; None, None = off."""
     lib = load_library()
     if start is None:
         lib.bebop_debug_set_timing_events(None, None)

@@ -1,8 +1,8 @@
 // General path of the verify step: works for any V, dtype and row stride the
 // C ABI admits.  Split-row fp32 sweeps (stats, then TV with the normalisers
 // known), a warp-per-sequence accept scan, and an fp64 inverse-CDF draw at the
-// stop row.  The wave kernel covers the common shapes faster and hands the
-// draws it cannot certify to the list-driven fp64 draw kernels of this file.
+// stop row.  The pipelined kernel (bebop_pipe.cu) covers the common shapes faster; this
+// path serves the remaining shapes, bebop_tv and the greedy mode.
 #include "bebop_kernels.h"
 
 namespace bebop {

@@ -44,15 +44,10 @@ cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft
 cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
                               const int* list, const int* count, cudaStream_t stream);
 
-// Wave kernel (bebop_wave.cu): persistent, ticket-scheduled, phases decoupled; same contract.
-bool wave_supported(const RowArgs& a);
-void wave_set_trace(long long* p);
-void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the wave kernel of the next calls (nullptr: off)
-cudaError_t wave_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                        cudaStream_t stream, bool* launched);
+void wave_set_trace(long long* p);                            // trace buffer of the main kernel (BEBOP_TRACE builds)
+void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the main kernel of the next calls (nullptr: off)
 
-// fp64 re-draw of the sequences a kernel listed (bebop_wave.cu); `w` is the wave workspace laid out by `wp`.
+// fp64 re-draw of the sequences a kernel listed (bebop_redraw.cu); `w` is the wave workspace laid out by `wp`.
 cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const int* fb_count,
                           const int* fb_list, char* w, const WavePlan& wp, cudaStream_t stream);
 void wave_flag_launch(const int* wait_failed, int32_t* row_status, int B, cudaStream_t stream);

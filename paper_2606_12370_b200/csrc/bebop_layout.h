@@ -6,12 +6,11 @@
 
 namespace bebop {
 
-// Workspace and schedule parameters of the wave kernel.
-constexpr int kWaveSliceVecs = 2048;   // 16-byte vectors per row slice, at most (wave kernel)
+// Workspace of the pipelined kernel and of the fp64 re-draw kernels.
 #ifndef BEBOP_PIPE_SLICE_VECS
 #define BEBOP_PIPE_SLICE_VECS 1536
 #endif
-constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // the same for the pipelined kernel (one stage of its ring)
+constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
 struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
     int wave_seqs, nwaves; // sequences per wave, waves
@@ -35,13 +34,13 @@ struct Plan {
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
     size_t off_fb;      // int [1 + B]: count and list of sequences whose draw goes to fp64
-    size_t off_wave;    // workspace of the wave kernel
+    size_t off_wave;    // workspace of the pipelined kernel
     size_t total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_cap = kWaveSliceVecs) {
+static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_cap = kPipeSliceVecs) {
     (void)dt;
     WavePlan w;
     w.T = (nvec + slice_cap - 1) / slice_cap; if (w.T < 1) w.T = 1;
@@ -55,7 +54,7 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.nwaves = (B + w.wave_seqs - 1) / w.wave_seqs;
     w.lag = 2;
     size_t o = 256;                                           // ticket, wait flag
-    w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per wave (wave kernel) or per sequence (pipelined kernel)
+    w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per sequence: rows merged
     w.off_adone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
@@ -100,8 +99,7 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
     {
-        const size_t w1 = make_wave_plan(B, K, p.nvec, dt).total, w2 = make_wave_plan(B, K, p.nvec, dt, kPipeSliceVecs).total;
-        p.off_wave = o;   o = align256(o + (w1 > w2 ? w1 : w2));
+        p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
     }
     p.total = o;
     return p;

@@ -1,5 +1,5 @@
-// Pipelined kernel: the wave schedule (see bebop_wave.cu) with the data movement and the task
-// bookkeeping taken off the compute warps.
+// Pipelined kernel: the hot path of bebop_verify as one persistent, ticket-scheduled kernel with the
+// data movement and the task bookkeeping taken off the compute warps.
 //
 // A CTA is eight consumer warps and one producer warp.  The producer's first lane draws tickets,
 // decodes them (step by step: tickets only grow), checks the wave's completion counter, fetches the
@@ -15,7 +15,7 @@
 // Every wait is bounded; a wait that gives up sets the wait flag (status bit 32 of every row).
 // No multicast, no cluster: each CTA copies from this GPU's own memory.
 #define BEBOP_CTA_SYNC() asm volatile("bar.sync 1, 256;" ::: "memory")
-#include "bebop_wave.cuh"
+#include "bebop_pipe.cuh"
 
 namespace bebop {
 

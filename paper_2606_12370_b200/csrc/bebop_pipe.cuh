@@ -1,0 +1,287 @@
+// Device code of the verify path that does not depend on how a CTA gets its data: workspace records,
+// small helpers, the residual arithmetic, the draw bound and phase D (the fast draw with its certificate).
+// The including file defines BEBOP_CTA_SYNC() (the barrier of the threads that run phase D) first.
+#pragma once
+#include "bebop_kernels.h"
+#include "bebop_ptx.cuh"
+
+#ifndef BEBOP_CTA_SYNC
+#error "define BEBOP_CTA_SYNC() before including bebop_pipe.cuh"
+#endif
+
+namespace bebop {
+
+namespace {
+
+constexpr int WT = 256;               // threads per CTA
+constexpr int WW = WT / 32;
+constexpr int SLICE_VECS = kPipeSliceVecs;   // vectors per row slice, at most
+constexpr int BEBOP_MAX_K_INT = 32;
+constexpr int MAX_SLICES = 64;
+constexpr int E_EMPTY = INT_MIN / 2;
+constexpr uint32_t kSpin = 1u << 22;
+
+struct __align__(16) P1Part { double s; int e; float m; };             // per (row, slice); m = NaN marks a non-finite logit
+struct __align__(16) RowStat { double inv_s; float ef; int e; int pad[2]; };   // per row, after the merge: 1/S, exponent E
+struct __align__(16) DPart { double tot; float sq; int pad; };        // per (sequence, slice)
+struct __align__(16) SeqInfo {          // per sequence, written by phase A
+    int n;                              // accept count (stop position); -1: fatal
+    int draw_row;                       // row whose residual is drawn from (n, or L for the bonus row); -1 none
+    int pad0;
+    int pad;
+};
+
+struct WaveArgs {
+    RowArgs r;
+    const int32_t* draft_tokens;
+    const float* u_accept;
+    const float* u_final;
+    VerifyOut o;
+    int* stop;
+    int* fb_count;
+    int* fb_list;
+    // workspace
+    int* ticket;          // [1]
+    int* wait_failed;     // [1]
+    int* p1done;          // [nwaves]
+    int* adone;           // [nwaves]
+    int* p2done;          // [nwaves]
+    int* rowcnt;          // [B][2K+1] pipelined kernel: softmax partials delivered per row
+    P1Part* part;         // [B][2K+1][T]
+    RowStat* rstat;       // [B][2K+1]
+    float* zpart;         // [B][K][T]
+    DPart* dpart;         // [B][T]
+    SeqInfo* sinfo;       // [B]
+    int ntickets, lag;
+    long long* trace;
+    int T, slice_vecs, wave_seqs, nwaves;
+};
+
+__device__ __forceinline__ float tau_of(const RowArgs& a, int b) { return a.temperature ? a.temperature[b] : a.temperature_all; }
+__device__ __forceinline__ bool tau_ok(float t) { return t > 0.f && t < INFINITY; }
+__device__ __forceinline__ int len_of(const RowArgs& a, int b) {
+    int L = a.draft_len ? a.draft_len[b] : a.K;
+    return max(0, min(L, a.K));
+}
+__device__ __forceinline__ int ld_acquire(const int* p) {
+    int v; asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
+}
+// Workspace records written by other CTAs of this launch are read through L2 only: the L1 of this SM
+// may hold an older copy of the line (a neighbouring record read earlier).
+template <typename T> __device__ __forceinline__ T ld_cg(const T* p) {
+    static_assert(sizeof(T) % 16 == 0, "16-byte records");
+    T r;
+#pragma unroll
+    for (int i = 0; i < (int)(sizeof(T) / 16); ++i)
+        reinterpret_cast<uint4*>(&r)[i] = __ldcg(reinterpret_cast<const uint4*>(p) + i);
+    return r;
+}
+__device__ __forceinline__ bool spin_ge(const int* p, int want) {
+    for (uint32_t i = 0; i < kSpin; ++i) {
+        if (ld_acquire(p) >= want) return true;
+        __nanosleep(64);
+    }
+    return false;
+}
+
+// The error bound a draw must clear.  The residual is formed from fp32 exponentials (ex2.approx:
+// 2 ulp), an fp32 argument (half an ulp of a number below 64, times 2^arg) and one fp32 rounding of
+// the product with the two-float normaliser, so each p, q carries a relative error below
+// delta = 2^-22; the errors of different tokens are independent, hence the error of a prefix sum is
+// of the order delta * sqrt(sum p^2 + q^2), and so is the part common to all tokens, the error of the
+// fp32-summed normalisers.  Measured on 40 000 draws with the certification switched off, the largest
+// error that changed a token was 0.1 * delta * sqrt(sum p^2 + q^2); kappa = 4 leaves a factor 40 over
+// that.
+#ifndef BEBOP_KAPPA
+#define BEBOP_KAPPA 4.0
+#endif
+__device__ __forceinline__ double draw_bound(double sumsq) {
+    const double delta = 2.384185791015625e-07;   // 2^-22
+    return BEBOP_KAPPA * delta * sqrt(sumsq) + 1e-300;
+}
+
+// c = log2(e) / tau in fp32, and 2^(x * c - E): the product is exact inside the fma, so the argument
+// carries one rounding of half an ulp of itself.  The rounding of c itself acts like a temperature
+// changed by at most 2^-24 relative; over a prefix of the vocabulary its effect, 2^-24 * sum p (z - zbar) / tau,
+// is a sum of zero-mean terms of the size draw_bound() already allows per token.
+struct TempScale { float hi; };
+__device__ __forceinline__ TempScale temp_scale(float tau) {
+    TempScale r; r.hi = kLog2e / (tau_ok(tau) ? tau : 1.f);
+    return r;
+}
+__device__ __forceinline__ float exp2_scaled(float x, const TempScale& t, float Ef) {
+    return ex2f(fmaf(x, t.hi, -Ef));
+}
+// E = ceil(m * c) of a maximum m, as int and float: any integer near m * c serves as the reference, and
+// integer references make every merge of partial sums an exact power-of-two scaling.
+__device__ __forceinline__ int ref_exponent(float m, const TempScale& t, float* Ef) {
+    const float th = fminf(fmaxf(m * t.hi, -4.0e6f), 4.0e6f);
+    return ceil_alu(th, Ef);
+}
+
+struct WaveShared {
+    float* vsum;                  // [slice_vecs / 2] per-vector residual mass (D phase); set by the kernel
+    double redd[WW];
+    float redf[2][WW];
+    int redi[WW];
+    int ticket, phase, wave, index;
+    // D-phase broadcast
+    double base, Ttarget, bound;
+    int owner_slice;
+};
+
+__device__ __forceinline__ const char* row_ptr(const RowArgs& R, int b, int r) {
+    // r in [0, K]: target row r; r in [K+1, 2K]: draft row r - (K+1)
+    const int K = R.K;
+    return r <= K ? R.target + ((int64_t)b * R.t_seq_rows + r) * R.t_row_bytes
+                  : R.draft + ((int64_t)b * R.d_seq_rows + (r - K - 1)) * R.d_row_bytes;
+}
+
+// residuals of one vector pair: p = 2^(x*c - E_p) / S_p, q likewise
+struct RowScale { float ef, inv, inv_lo; };     // exponent E; 1/S = inv + inv_lo to about 2^-48
+__device__ __forceinline__ RowScale row_scale(const RowStat& s) {
+    RowScale r; r.ef = s.ef; r.inv = (float)s.inv_s; r.inv_lo = (float)(s.inv_s - (double)r.inv);
+    return r;
+}
+__device__ __forceinline__ RowScale no_row() { RowScale r; r.ef = 0.f; r.inv = 0.f; r.inv_lo = 0.f; return r; }
+
+// FINE (the rows a token is drawn from): the normaliser enters as two floats, so that its rounding to fp32
+// is not an error common to all tokens of the row; what is left is one rounding per token.
+template <int DT, bool FINE>
+__device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, bool pair, const TempScale& c, const RowScale& P,
+                                             const RowScale& Q, float* r, float* sq) {
+    constexpr int VEC = Elem<DT>::VEC;
+    float fp[VEC], fq[VEC];
+    unpack<DT>(rp, fp);
+    if (pair) unpack<DT>(rq, fq);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        const float ap = exp2_scaled(fp[i], c, P.ef);
+        const float aq = pair ? exp2_scaled(fq[i], c, Q.ef) : 0.f;
+        // explicit roundings: a contracted p - a*inv would leave rounding dust when the rows are equal
+        const float p = FINE ? __fmaf_rn(ap, P.inv_lo, __fmul_rn(ap, P.inv)) : __fmul_rn(ap, P.inv);
+        const float q = pair ? (FINE ? __fmaf_rn(aq, Q.inv_lo, __fmul_rn(aq, Q.inv)) : __fmul_rn(aq, Q.inv)) : 0.f;
+        r[i] = fmaxf(p - q, 0.f);
+        if (sq) { *sq = fmaf(p, p, *sq); *sq = fmaf(q, q, *sq); }
+    }
+}
+
+// ------------------------------------------------------------------ phase D
+template <int DT>
+__device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b) {
+    constexpr int VEC = Elem<DT>::VEC;
+    const RowArgs& R = a.r;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1, T = 2 * a.T, sv = a.slice_vecs >> 1;
+    const SeqInfo si = ld_cg(a.sinfo + b);
+    if (si.n < 0) return;
+    // TV of every draft position: slice parts in slice order
+    if (tid < L && a.o.tv) {
+        float z = 0.f;
+        for (int s = 0; s < T; ++s) z += __ldcg(a.zpart + ((int64_t)b * K + tid) * T + s);
+        a.o.tv[(int64_t)b * K + tid] = fminf(fmaxf(z, 0.f), 1.f);
+    }
+    const int k = si.draw_row;
+    if (k < 0) return;
+    const bool pair = k < L;
+    if (tid == 0) {
+        double Z = 0.0, sumsq = 0.0;
+        for (int s = 0; s < T; ++s) { const DPart dp = ld_cg(a.dpart + (int64_t)b * T + s); Z += dp.tot; sumsq += (double)dp.sq; }
+        const double Tt = (double)a.u_final[b] * Z;
+        double run = 0.0; int owner = -1; double base = 0.0;
+        for (int s = 0; s < T; ++s) {
+            const double nx = run + ld_cg(a.dpart + (int64_t)b * T + s).tot;
+            if (owner < 0 && Tt > run && Tt <= nx) { owner = s; base = run; }
+            run = nx;
+        }
+        S.owner_slice = (Tt > 0.0) ? owner : -1;
+        S.base = base; S.Ttarget = Tt; S.bound = draw_bound(sumsq);
+    }
+    BEBOP_CTA_SYNC();
+    const int s = S.owner_slice;
+    int found_y = -1, found_cert = 0;
+    if (s >= 0) {
+        const float tau = tau_of(R, b);
+        const TempScale c = temp_scale(tau);
+        const RowScale SP = row_scale(ld_cg(a.rstat + (int64_t)b * NR + k));
+        RowScale SQ = no_row();
+        if (pair) SQ = row_scale(ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k));
+        const int v0 = s * sv;
+        const int nv = max(min(sv, R.nvec - v0), 0);
+        const char* prow = row_ptr(R, b, k) + (int64_t)v0 * 16;
+        const char* qrow = pair ? row_ptr(R, b, K + 1 + k) + (int64_t)v0 * 16 : nullptr;
+        // per-vector residual mass, same arithmetic as phase P2
+        for (int v = tid; v < nv; v += WT) {
+            uint4 rp = ldg16(prow + (size_t)v * 16), rq = neg_inf_vec<DT>();
+            if (pair) rq = ldg16(qrow + (size_t)v * 16);
+            const int gbase = (v0 + v) * VEC;
+            if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
+            float r[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
+            S.vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+        }
+        BEBOP_CTA_SYNC();
+        // contiguous ranges of vectors per thread, inclusive scan over threads
+        const int per = (nv + WT - 1) / WT;
+        const int vb = min(tid * per, nv), ve = min(vb + per, nv);
+        double mine = 0.0;
+        for (int v = vb; v < ve; ++v) mine += (double)S.vsum[v];
+        double incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { double t2 = shfl_up_d(incl, d); if (lane >= d) incl += t2; }
+        if (lane == 31) S.redd[warp] = incl;
+        BEBOP_CTA_SYNC();
+        double woff = 0.0;
+        for (int w = 0; w < warp; ++w) woff += S.redd[w];
+        double prev = shfl_up_d(incl, 1);
+        if (lane == 0) prev = 0.0;
+        const double Tt = S.Ttarget, bound = S.bound;
+        const double lower = S.base + woff + prev, upper = S.base + woff + incl;
+        if (lower < Tt && Tt <= upper) {
+            double C = lower;
+            for (int v = vb; v < ve && found_y < 0; ++v) {
+                const double nxt = C + (double)S.vsum[v];
+                if (Tt <= nxt) {
+                    uint4 rp = ldg16(prow + (size_t)v * 16), rq = neg_inf_vec<DT>();
+                    if (pair) rq = ldg16(qrow + (size_t)v * 16);
+                    const int gbase = (v0 + v) * VEC;
+                    if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
+                    float r[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                    residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
+                    double Cw = C;
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        if (found_y < 0) {
+                            const double r1 = (double)r[i];
+                            const double Cn = Cw + r1;
+                            if (r1 > 0.0 && Cn >= Tt) { found_y = gbase + i; found_cert = (Tt - Cw > bound) && (Cn - Tt >= bound); }
+                            Cw = Cn;
+                        }
+                    }
+                    break;
+                }
+                C = nxt;
+            }
+        }
+    }
+    // at most one thread should have found the token
+    const unsigned own = __ballot_sync(0xffffffffu, found_y >= 0);
+    if (lane == 0) S.redi[warp] = -1;
+    BEBOP_CTA_SYNC();
+    if (own && lane == (__ffs(own) - 1)) S.redi[warp] = (__popc(own) == 1 && found_cert) ? found_y : -2;
+    BEBOP_CTA_SYNC();
+    if (tid == 0) {
+        int y = -1, cnt = 0;
+        for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
+        if (cnt == 1 && y >= 0) a.o.out_tokens[(int64_t)b * (K + 1) + k] = y;
+        else { int idx = atomicAdd(a.fb_count, 1); a.fb_list[idx] = b; }
+    }
+}
+
+}  // namespace
+
+}  // namespace bebop

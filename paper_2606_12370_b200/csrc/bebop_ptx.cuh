@@ -1,4 +1,4 @@
-// Device helpers of the wave kernel: warp reductions through redux, order-preserving
+// Device helpers of the pipelined kernel: warp reductions through redux, order-preserving
 // float/int map, packed bf16 maximum, power-of-two construction, conversion-free ceil.
 #pragma once
 #include <cuda_runtime.h>
