@@ -17,7 +17,7 @@ struct WavePlan {
     int lag;               // waves of stats work scheduled between a phase and the phase it depends on
     size_t off_p1done, off_adone, off_p2done, off_xdone, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
-    size_t off_part, off_rstat, off_zpart, off_dpart, off_sinfo, total;
+    size_t off_part, off_rstat, off_dpart, off_tvacc, off_sinfo, total;
 };
 
 struct Plan {
@@ -59,13 +59,14 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_rowcnt = o; o += align256(sizeof(int) * (size_t)B * NR);
+    // records that readers validate by a mark inside them, and sums that start from zero
+    w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
+    w.off_rstat = o;  o += align256(16 * (size_t)B * NR);
+    w.off_dpart = o;  o += align256(16 * (size_t)B * 2 * w.T);
+    w.off_tvacc = o;  o += align256(8 * (size_t)B * (K > 0 ? K : 1));
     w.zero_bytes = o;
     w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);
     w.off_xmass = o;  o += align256(8 * (size_t)B * 4 * w.T * 8);
-    w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
-    w.off_rstat = o;  o += align256(32 * (size_t)B * NR);
-    w.off_zpart = o;  o += align256(4 * (size_t)B * (K > 0 ? K : 1) * 2 * w.T);
-    w.off_dpart = o;  o += align256(16 * (size_t)B * 2 * w.T);
     w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.total = o;
     return w;

@@ -38,6 +38,8 @@ constexpr int kPend = 4;                          // runs a producer may set asi
 #define BEBOP_PIPE_BATCH 2
 #endif
 constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time
+constexpr double kFixTv = 1099511627776.0;             // 2^40: fixed point of TV parts and sums of squares
+constexpr double kFixMass = 288230376151711744.0;      // 2^58: fixed point of the draw-row mass
 constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
 
 struct __align__(16) TaskDesc {
@@ -283,8 +285,13 @@ __device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) 
     P1Part mine[2];
     int cnt = 0;
     for (int s = lane; s < T && cnt < 2; s += 32) {
-        mine[cnt] = ld_cg(pp + s); e_l = max(e_l, mine[cnt].e);
-        if (mine[cnt].m != mine[cnt].m) f_l = 1;
+        // the record's exponent is stored as 2e + 1: zero means the record is not there yet
+        P1Part rec = ld_cg(pp + s);
+        for (uint32_t i = 0; rec.e == 0 && i < kSpin; ++i) { __nanosleep(64); rec = ld_cg(pp + s); }
+        if (rec.e == 0) atomicExch(a.wait_failed, 1);
+        rec.e = (rec.e - 1) >> 1;
+        mine[cnt] = rec; e_l = max(e_l, rec.e);
+        if (rec.m != rec.m) f_l = 1;
         cnt++;
     }
     const int Em = redux_max(e_l);
@@ -294,8 +301,8 @@ __device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) 
     if (lane == 0) {
         int st = 0;
         if (f_l || !(s_l == s_l)) st = ST_NONFINITE; else if (Em == E_EMPTY) st = ST_EMPTY;
-        RowStat rs; rs.inv_s = (!st && s_l > 0.0) ? 1.0 / s_l : 0.0; rs.ef = (float)Em; rs.e = Em; rs.pad[0] = st; rs.pad[1] = 0;
-        a.rstat[(int64_t)b * NR + r] = rs;
+        RowStat rs; rs.inv_s = (!st && s_l > 0.0) ? 1.0 / s_l : 0.0; rs.e = Em; rs.st = st | kRowValid;
+        st16(a.rstat + (int64_t)b * NR + r, rs);
     }
 }
 
@@ -312,17 +319,24 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     const int tk = active ? a.draft_tokens[(int64_t)b * K + lane] : 0;
     const float u = active ? a.u_accept[(int64_t)b * K + lane] : 0.f;
     RowStat sp, sq, sb;
-    sp.inv_s = 0.0; sp.ef = 0.f; sp.e = E_EMPTY; sp.pad[0] = 0; sp.pad[1] = 0;
+    sp.inv_s = 0.0; sp.e = E_EMPTY; sp.st = 0;
     sq = sp;
-    if (active) { sp = ld_cg(a.rstat + (int64_t)b * NR + lane); sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + lane); }
-    sb = ld_cg(a.rstat + (int64_t)b * NR + L);                         // bonus row (row L <= K: always merged)
+    auto row = [&](int r) {                                            // a merged row's record (waits, bounded, for its mark)
+        RowStat x = ld_cg(a.rstat + (int64_t)b * NR + r);
+        for (uint32_t i = 0; x.st == 0 && i < kSpin; ++i) { __nanosleep(64); x = ld_cg(a.rstat + (int64_t)b * NR + r); }
+        if (x.st == 0) atomicExch(a.wait_failed, 1);
+        x.st &= 0xff;
+        return x;
+    };
+    if (active) { sp = row(lane); sq = row(K + 1 + lane); }
+    sb = row(L);                                                       // bonus row (row L <= K: always merged)
     int seq_st = ok ? 0 : ST_BAD_TEMP;
     const bool tok_ok = tk >= 0 && tk < V;
     float zpx = 0.f, zqx = 0.f;
     if (active && tok_ok) { zpx = load_one<DT>(row_ptr(R, b, lane), tk); zqx = load_one<DT>(row_ptr(R, b, K + 1 + lane), tk); }
     if (!seq_st && __ballot_sync(0xffffffffu, active && !tok_ok)) seq_st = ST_BAD_TOKEN;
     // the first bad row pair decides the status; rows after it do not count
-    const int rs = active ? (sp.pad[0] | sq.pad[0]) : 0;
+    const int rs = active ? (sp.st | sq.st) : 0;
     const unsigned badrows = __ballot_sync(0xffffffffu, rs != 0);
     const int first_bad = badrows ? __ffs(badrows) - 1 : 32;
     const int rs_first = __shfl_sync(0xffffffffu, rs, first_bad & 31);
@@ -337,7 +351,7 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     }
     const unsigned rej = __ballot_sync(0xffffffffu, active && !acc);
     const int n = rej ? __ffs(rej) - 1 : L;
-    if (!(seq_st & ST_FATAL) && n == L && sb.pad[0]) seq_st |= sb.pad[0];   // bonus row, counted only now
+    if (!(seq_st & ST_FATAL) && n == L && sb.st) seq_st |= sb.st;   // bonus row, counted only now
     const bool fatal = (seq_st & ST_FATAL) != 0;
     const int nn = fatal ? 0 : n;
     // outputs: lane q writes position q (position nn is filled by the draw)
@@ -364,10 +378,8 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
 // Each consumer warp leaves its partial of a task in shared memory and signals the stage's `pdone` barrier;
 // the publisher warp merges the eight partials in warp order and publishes the result, off the consumers'
 // path.
-__device__ __forceinline__ int add_acq_rel(int* p, int v) {
-    int old;
-    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-    return old;
+__device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
 }
 
 // P1: softmax partial (E, S) of one slice of one row, from shared memory.
@@ -537,17 +549,17 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
             for (int k = 0; k < WW; ++k) { sum += __shfl_sync(0xffffffffu, mine, k); mc = max_nan(mc, __shfl_sync(0xffffffffu, f1, k)); }
             int run_a = 0;
             if (lane == 0) {
-                P1Part p; p.s = (mc != mc) ? 0.0 : sum; p.e = Ec; p.m = mc;
-                a.part[((int64_t)b * (2 * K + 1) + r) * a.T + sl] = p;
-                // the last softmax partial of a row starts the merge of that row (release: the partial above;
-                // acquire: the partials of the other slices)
-                run_a = add_acq_rel(&a.rowcnt[(int64_t)b * (2 * K + 1) + r], 1) == a.T - 1;
+                // the slice's record (exponent stored as 2e + 1: zero means "not there yet"), then the row's counter.
+                // No fence: whoever the counter wakes checks every record's mark before using it.
+                P1Part p; p.s = (mc != mc) ? 0.0 : sum; p.e = 2 * Ec + 1; p.m = mc;
+                st16(a.part + ((int64_t)b * (2 * K + 1) + r) * a.T + sl, p);
+                run_a = atomicAdd(&a.rowcnt[(int64_t)b * (2 * K + 1) + r], 1) == a.T - 1;
             }
             if (__shfl_sync(0xffffffffu, run_a, 0)) {
                 merge_row_warp(a, b, r);
                 // the last merged row of the sequence (2L+1 rows are in use) starts the accept scan
                 int last_row = 0;
-                if (lane == 0) last_row = add_acq_rel(&a.p1done[b], 1) == 2 * len_of(R, b);
+                if (lane == 0) last_row = atomicAdd(&a.p1done[b], 1) == 2 * len_of(R, b);
                 if (__shfl_sync(0xffffffffu, last_row, 0)) accept_warp<DT>(a, b);
             }
         } else {
@@ -557,9 +569,15 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
                 zz += __shfl_sync(0xffffffffu, f0, k); sq += __shfl_sync(0xffffffffu, f1, k); tot += __shfl_sync(0xffffffffu, dd, k);
             }
             if (lane == 0) {
-                if (flags & 1) a.zpart[((int64_t)b * K + r) * T2 + sl] = zz;
-                if (flags & 2) { DPart dp; dp.tot = tot; dp.sq = sq; dp.pad = 0; a.dpart[(int64_t)b * T2 + sl] = dp; }
-                release_add(&a.p2done[b]);
+                // Fixed point with a count of one in the low bits of the same word: one relaxed add publishes value
+                // and count together, and integer sums do not depend on the order of arrival.
+                if (flags & 1) red_add_u64(a.tvacc + (int64_t)b * K + r, ((unsigned long long)__double2ll_rn((double)zz * kFixTv) << 16) | 1ull);
+                if (flags & 2) {
+                    unsigned long long* wd = a.dacc + ((int64_t)b * T2 + sl) * 2;
+                    red_add_u64(wd, ((unsigned long long)__double2ll_rn(tot * kFixMass) << 4) | 1ull);
+                    red_add_u64(wd + 1, ((unsigned long long)__double2ll_rn((double)sq * kFixTv) << 4) | 1ull);
+                }
+                asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" :: "l"(a.p2done + b) : "memory");
             }
         }
     }
@@ -600,8 +618,8 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (d.phase == 0) pipe_p1<DT>(a, S, d, sd, stage, it);
         else if (d.phase == 2) pipe_p2<DT>(a, S, d, sd, stage, it);
         else {
-            if (tid == 0) S.W.vsum = reinterpret_cast<float*>(data + (size_t)stage * STAGE_BYTES);   // a D task's stage holds no logits
-            phase_d<DT>(a, S.W, d.b);
+            // a D task's stage holds no logits: it is the task's scratch (per-vector masses, slice masses)
+            phase_d<DT>(a, S.W, d.b, reinterpret_cast<float*>(data + (size_t)stage * STAGE_BYTES));
             BEBOP_CTA_SYNC();
 
         }
@@ -677,8 +695,8 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.rowcnt = reinterpret_cast<int*>(w + wp.off_rowcnt);
     wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
     wa.rstat = reinterpret_cast<RowStat*>(w + wp.off_rstat);
-    wa.zpart = reinterpret_cast<float*>(w + wp.off_zpart);
-    wa.dpart = reinterpret_cast<DPart*>(w + wp.off_dpart);
+    wa.dacc = reinterpret_cast<unsigned long long*>(w + wp.off_dpart);
+    wa.tvacc = reinterpret_cast<unsigned long long*>(w + wp.off_tvacc);
     wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
     wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;

@@ -22,7 +22,15 @@ constexpr int E_EMPTY = INT_MIN / 2;
 constexpr uint32_t kSpin = 1u << 22;
 
 struct __align__(16) P1Part { double s; int e; float m; };             // per (row, slice); m = NaN marks a non-finite logit
-struct __align__(16) RowStat { double inv_s; float ef; int e; int pad[2]; };   // per row, after the merge: 1/S, exponent E
+struct __align__(16) RowStat { double inv_s; int e; int st; };   // per row, after the merge: 1/S, exponent E, status bits | kRowValid
+constexpr int kRowValid = 0x100;
+// One 16-byte store of a 16-byte record: a reader that sees the record's validity mark sees all of it.  The
+// records that CTAs pass to each other start at zero and carry such a mark, so they need no fence.
+template <typename T> __device__ __forceinline__ void st16(T* p, const T& v) {
+    static_assert(sizeof(T) == 16, "16-byte record");
+    const uint4 b = *reinterpret_cast<const uint4*>(&v);
+    asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" :: "l"(p), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
 struct __align__(16) DPart { double tot; float sq; int pad; };        // per (sequence, slice)
 struct __align__(16) SeqInfo {          // per sequence, written by phase A
     int n;                              // accept count (stop position); -1: fatal
@@ -49,8 +57,8 @@ struct WaveArgs {
     int* rowcnt;          // [B][2K+1] pipelined kernel: softmax partials delivered per row
     P1Part* part;         // [B][2K+1][T]
     RowStat* rstat;       // [B][2K+1]
-    float* zpart;         // [B][K][T]
-    DPart* dpart;         // [B][T]
+    unsigned long long* dacc;    // [B][2T][2] draw-row mass (2^-58) and sum of squares (2^-40), each << 4 | parts added
+    unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
     int ntickets, lag;
     long long* trace;
@@ -120,7 +128,6 @@ __device__ __forceinline__ int ref_exponent(float m, const TempScale& t, float* 
 }
 
 struct WaveShared {
-    float* vsum;                  // [slice_vecs / 2] per-vector residual mass (D phase); set by the kernel
     double redd[WW];
     float redf[2][WW];
     int redi[WW];
@@ -140,7 +147,7 @@ __device__ __forceinline__ const char* row_ptr(const RowArgs& R, int b, int r) {
 // residuals of one vector pair: p = 2^(x*c - E_p) / S_p, q likewise
 struct RowScale { float ef, inv, inv_lo; };     // exponent E; 1/S = inv + inv_lo to about 2^-48
 __device__ __forceinline__ RowScale row_scale(const RowStat& s) {
-    RowScale r; r.ef = s.ef; r.inv = (float)s.inv_s; r.inv_lo = (float)(s.inv_s - (double)r.inv);
+    RowScale r; r.ef = (float)s.e; r.inv = (float)s.inv_s; r.inv_lo = (float)(s.inv_s - (double)r.inv);
     return r;
 }
 __device__ __forceinline__ RowScale no_row() { RowScale r; r.ef = 0.f; r.inv = 0.f; r.inv_lo = 0.f; return r; }
@@ -167,8 +174,24 @@ __device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, b
 }
 
 // ------------------------------------------------------------------ phase D
+// mass and sum of squares of half slice i of a sequence's draw rows (waits, bounded, for a part not there yet)
+__device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
+    unsigned long long w0 = 0, w1 = 0;
+    for (uint32_t k = 0; k < kSpin; ++k) {
+        w0 = __ldcg(a.dacc + 2 * i); w1 = __ldcg(a.dacc + 2 * i + 1);
+        if ((w0 & 15ull) != 0 && (w1 & 15ull) != 0) break;
+        __nanosleep(64);
+    }
+    if ((w0 & 15ull) == 0 || (w1 & 15ull) == 0) atomicExch(a.wait_failed, 1);
+    DPart d;
+    d.tot = (double)(w0 >> 4) * 3.469446951953614e-18;            // 2^-58
+    d.sq = (float)((double)(w1 >> 4) * 9.094947017729282e-13);    // 2^-40
+    d.pad = 1;
+    return d;
+}
+constexpr int NTH_D = WT;            // threads that run phase D
 template <int DT>
-__device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b) {
+__device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b, float* vsum) {
     constexpr int VEC = Elem<DT>::VEC;
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -178,19 +201,32 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
     // TV of every draft position: slice parts in slice order
     if (tid < L && a.o.tv) {
         float z = 0.f;
-        for (int s = 0; s < T; ++s) z += __ldcg(a.zpart + ((int64_t)b * K + tid) * T + s);
+        // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
+        unsigned long long w = 0;
+        for (uint32_t i = 0; i < kSpin; ++i) {
+            w = __ldcg(a.tvacc + (int64_t)b * K + tid);
+            if ((int)(w & 0xffffull) >= T) break;
+            __nanosleep(64);
+        }
+        if ((int)(w & 0xffffull) < T) atomicExch(a.wait_failed, 1);
+        z = (float)((double)(w >> 16) * 9.094947017729282e-13);      // 2^-40
         a.o.tv[(int64_t)b * K + tid] = fminf(fmaxf(z, 0.f), 1.f);
     }
     const int k = si.draw_row;
     if (k < 0) return;
     const bool pair = k < L;
+    // the half slices' masses: one thread each fetches its slice's words (in parallel), thread 0 then scans them
+    double* dtot = reinterpret_cast<double*>(vsum + SLICE_VECS / 2);     // behind the per-vector masses
+    float* dsq = reinterpret_cast<float*>(dtot + 2 * MAX_SLICES);
+    for (int s = tid; s < T; s += NTH_D) { const DPart dp = load_dpart(a, (int64_t)b * T + s); dtot[s] = dp.tot; dsq[s] = dp.sq; }
+    BEBOP_CTA_SYNC();
     if (tid == 0) {
         double Z = 0.0, sumsq = 0.0;
-        for (int s = 0; s < T; ++s) { const DPart dp = ld_cg(a.dpart + (int64_t)b * T + s); Z += dp.tot; sumsq += (double)dp.sq; }
+        for (int s = 0; s < T; ++s) { Z += dtot[s]; sumsq += (double)dsq[s]; }
         const double Tt = (double)a.u_final[b] * Z;
         double run = 0.0; int owner = -1; double base = 0.0;
         for (int s = 0; s < T; ++s) {
-            const double nx = run + ld_cg(a.dpart + (int64_t)b * T + s).tot;
+            const double nx = run + dtot[s];
             if (owner < 0 && Tt > run && Tt <= nx) { owner = s; base = run; }
             run = nx;
         }
@@ -220,14 +256,14 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
 #pragma unroll
             for (int i = 0; i < 8; ++i) r[i] = 0.f;
             residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
-            S.vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+            vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
         }
         BEBOP_CTA_SYNC();
         // contiguous ranges of vectors per thread, inclusive scan over threads
         const int per = (nv + WT - 1) / WT;
         const int vb = min(tid * per, nv), ve = min(vb + per, nv);
         double mine = 0.0;
-        for (int v = vb; v < ve; ++v) mine += (double)S.vsum[v];
+        for (int v = vb; v < ve; ++v) mine += (double)vsum[v];
         double incl = mine;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) { double t2 = shfl_up_d(incl, d); if (lane >= d) incl += t2; }
@@ -242,7 +278,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b)
         if (lower < Tt && Tt <= upper) {
             double C = lower;
             for (int v = vb; v < ve && found_y < 0; ++v) {
-                const double nxt = C + (double)S.vsum[v];
+                const double nxt = C + (double)vsum[v];
                 if (Tt <= nxt) {
                     uint4 rp = ldg16(prow + (size_t)v * 16), rq = neg_inf_vec<DT>();
                     if (pair) rq = ldg16(qrow + (size_t)v * 16);
