@@ -1,16 +1,26 @@
 // Pipelined kernel: the hot path of bebop_verify as one persistent, ticket-scheduled kernel with the
-// data movement and the task bookkeeping taken off the compute warps.
+// data movement and the bookkeeping taken off the compute warps.
 //
-// A CTA is eight consumer warps and one producer warp.  The producer's first lane draws tickets,
-// decodes them (step by step: tickets only grow), checks the wave's completion counter, fetches the
-// few per-task numbers (length, temperature, row normalisers) and, once a stage of the shared-memory
-// ring is free, describes the task there and starts bulk copies (cp.async.bulk, completion counted
-// on the stage's mbarrier) of the slice of logits the task reads: one slice of one row for P1, the
-// same half slice of the target and the draft row for P2, nothing for A and D.  The consumers wait
-// on the stage's barrier, compute from shared memory, and hand the stage back.  A task's partial
-// result is merged by whichever warp finishes last (a shared counter; the merge reads the eight warp
-// partials in warp order, so the result does not depend on who was last), which also publishes it
-// and bumps the wave's completion counter: no CTA-wide barrier sits on the streaming path.
+// The work is a queue of tickets in three blocks: P1 (softmax partial of one slice of one row) for
+// every row, then P2 (TV and residual mass of one half slice of a row pair) for every position, then D
+// (the fast draw with its certificate) for every sequence; sequences ascending.  Phase A -- merging a
+// row's partials, and the accept scan of a sequence -- has no tickets: it runs in the publisher warp
+// that completes the row / the sequence, long before the second sweep asks for its results.
+//
+// A CTA is eight consumer warps, a producer warp and a publisher warp around a ring of shared-memory
+// stages.  The producer's first lane claims tickets, decodes them into runs of consecutive slices,
+// fetches the few per-row numbers (length, temperature, row normalisers), checks that the sequence is
+// ready for the phase (a run that is not is set aside while later tickets go ahead) and, once a stage
+// is free, describes the task there and starts bulk copies (cp.async.bulk, completion counted on the
+// stage's mbarrier) of the logits the task reads.  The consumers wait on the stage's barrier, compute
+// from shared memory, leave one partial per warp and signal a second barrier; the publisher takes the
+// eight partials, hands the stage back, merges them in warp order and publishes.  No CTA-wide barrier
+// sits on the streaming path.
+//
+// What CTAs pass to each other through global memory needs no fence: 16-byte records written by one
+// store and carrying a validity mark (the memory starts at zero), and fixed-point sums with a count of
+// contributions in the low bits of the same word, added by relaxed atomics.  Counters only say when to
+// look; whoever looks checks the marks and waits (bounded) for a record that is not there yet.
 //
 // Every wait is bounded; a wait that gives up sets the wait flag (status bit 32 of every row).
 // No multicast, no cluster: each CTA copies from this GPU's own memory.
@@ -37,7 +47,11 @@ constexpr int kPend = 4;                          // runs a producer may set asi
 #ifndef BEBOP_PIPE_BATCH
 #define BEBOP_PIPE_BATCH 2
 #endif
-constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time
+constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time in the first sweep
+#ifndef BEBOP_PIPE_BATCH2
+#define BEBOP_PIPE_BATCH2 2
+#endif
+constexpr int kBatch2 = BEBOP_PIPE_BATCH2;        // ... and in the second sweep (more per-row numbers to fetch)
 constexpr double kFixTv = 1099511627776.0;             // 2^40: fixed point of TV parts and sums of squares
 constexpr double kFixMass = 288230376151711744.0;      // 2^58: fixed point of the draw-row mass
 constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
@@ -65,6 +79,7 @@ struct PipeShared {
     double wd[NST][WW];
     int wi[NST][WW];
     Run pend[kPend];                            // producer: runs set aside
+    int logn;                                   // trace builds: events logged
 #ifdef BEBOP_TRACE
     long long t_empty[NST];
 #endif
@@ -113,6 +128,13 @@ __device__ __forceinline__ void tl_max(const WaveArgs& a, int w, int i) { if (a.
 #define TL_MAX(w, i) do { } while (0)
 #endif
 
+#ifdef BEBOP_TRACE
+// event log of one CTA: (clock, code * 1e6 + task number)
+#define PLOG(code, n) do { if (blockIdx.x == 5 && a.trace) { const int k_ = atomicAdd(&S.logn, 1); if (k_ < 3000) { a.trace[2048 + 2 * k_] = clock64(); a.trace[2049 + 2 * k_] = (long long)(code) * 1000000 + (n); } } } while (0)
+#else
+#define PLOG(code, n) do { } while (0)
+#endif
+
 // ------------------------------------------------------------------ producer
 // One thread.  Tickets are claimed kBatch at a time; consecutive tickets of one (phase, wave) block are
 // consecutive slices of a row, then the next row, then the next sequence, so a batch decodes once and
@@ -157,7 +179,8 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     int npend = 0;
     bool exhausted = false;
     int bt = 0, bleft = 0;                         // tickets of the claimed batch not yet turned into runs
-    int next = atomicAdd(a.ticket, kBatch);
+    int next_cnt = kBatch;                         // tickets of the claim in flight (more at a time in the second sweep)
+    int next = atomicAdd(a.ticket, next_cnt);
     int it = 0;
     for (;;) {
         // ---- next run
@@ -169,9 +192,9 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             for (int i = 0; i < npend; ++i) S.pend[i] = S.pend[i + 1];
         } else {
             if (bleft == 0 && !exhausted) {
-                bt = next; bleft = min(kBatch, a.ntickets - bt);
+                bt = next; bleft = min(next_cnt, a.ntickets - bt);
                 if (bleft <= 0) { bleft = 0; exhausted = true; }
-                else next = atomicAdd(a.ticket, kBatch);
+                else { next_cnt = bt + bleft >= n1 ? kBatch2 : kBatch; next = atomicAdd(a.ticket, next_cnt); }
             }
             if (bleft == 0) {
                 if (npend > 0) continue;
@@ -252,6 +275,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                     if (a.trace && blockIdx.x == 5 && it < 100) { a.trace[2048 + it * 20] = q1_; a.trace[2048 + it * 20 + 17] = ph; }
 #endif
                     S.desc[stage] = d;
+                    PLOG(1 + 10 * ph, it);
                     const uint32_t bytes = (uint32_t)d.nv * 16u;
                     if (row0 && bytes) {
                         mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
@@ -593,6 +617,7 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     const int tid = threadIdx.x;
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], WW + 1); mbar_init(&S.pdone[i], WW); }
+        S.logn = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -611,6 +636,7 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (!mbar_wait(&S.full[stage], par)) { if (tid == 0) atomicExch(a.wait_failed, 1); break; }
         const TaskDesc d = S.desc[stage];
         if (d.phase < 0) break;
+        if (tid == 0) PLOG(2, it);
 #ifdef BEBOP_TRACE
         const long long c1_ = clock64();
 #endif
