@@ -64,10 +64,10 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.off_rstat = o;  o += align256(16 * (size_t)B * NR);
     w.off_dpart = o;  o += align256(16 * (size_t)B * 2 * w.T);
     w.off_tvacc = o;  o += align256(8 * (size_t)B * (K > 0 ? K : 1));
+    w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.zero_bytes = o;
     w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);
     w.off_xmass = o;  o += align256(8 * (size_t)B * 4 * w.T * 8);
-    w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.total = o;
     return w;
 }

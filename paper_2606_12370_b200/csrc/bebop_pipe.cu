@@ -147,10 +147,8 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     const int B = R.B;
     const int c0 = NR * T, c2 = (K + 1) * T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
-    // Ticket order: all of P1 (sequences ascending), then all of P2 and then all of D with the sequences
-    // DESCENDING: the last sequences P1 streamed are the ones still in L2 when P2 begins.  Every logit comes
-    // from DRAM once per sweep except that tail.  Phase A has no tickets: it runs in the warp that
-    // completes a sequence's last softmax partial, long before P2 asks for it.
+    // Ticket order: all of P1, then all of P2, then all of D, sequences ascending: the first sequences' accept
+    // scans are long done when the second sweep starts.  Every logit comes from DRAM once per sweep.
     const int n1 = B * c0, n2 = B * c2;
     // the run of block-consecutive tasks that starts at ticket t and has at most `want` tasks
     auto decode = [&](int t, int want) {
@@ -166,8 +164,14 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     // Is sequence b ready for the phase?  P2 needs its accept scan, D all of its P2 partials.  A run that is
     // not ready is set aside (up to kPend of them) while later tickets go ahead; the oldest one is looked at
     // again before every new run and waited for only when the shelf is full or no tickets are left.
+    // the sequence's record of the accept scan, valid once its mark is set (waits, bounded, if asked to)
+    auto seq_info = [&](int b, bool wait) {
+        SeqInfo si = ld_cg(a.sinfo + b);
+        if (wait) for (uint32_t i = 0; si.pad == 0 && i < kSpin; ++i) { __nanosleep(64); si = ld_cg(a.sinfo + b); }
+        return si;
+    };
     auto ready = [&](int ph, int b, bool wait) {
-        if (ph == 2) return wait ? spin_ge(&a.adone[b], 1) : ld_acquire(&a.adone[b]) >= 1;
+        if (ph == 2) return seq_info(b, wait).pad != 0;
         if (ph == 3) return wait ? spin_ge(&a.p2done[b], c2) : ld_acquire(&a.p2done[b]) >= c2;
         return true;
     };
@@ -204,11 +208,14 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 mbar_arrive(&S.full[stage]);
                 return;
             }
+            PLOG(20, bt);
             run = decode(bt, bleft);
             // a P2 or D run stays within one sequence, so that one readiness check covers it
             if (run.ph == 2) run.cnt = min(run.cnt, c2 - run.off % c2); else if (run.ph == 3) run.cnt = 1;
             bt += run.cnt; bleft -= run.cnt;
-            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; continue; }
+            PLOG(21, run_seq(run));
+            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; PLOG(22, run_seq(run)); continue; }
+            PLOG(23, run_seq(run));
         }
         // ---- the tasks of the run
         const int ph = run.ph, wv = 0;
@@ -232,26 +239,30 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 skip = is_target ? k > L : k >= L;
                 row0 = row_ptr(R, b, r);
             } else if (ph == 2) {
-                const int k = r, L = len_of(R, b);
+                // everything the row needs is requested at once (the sequence was seen ready: its records are there)
+                const int k = r;
+                const SeqInfo si = ld_cg(a.sinfo + b);
+                RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
+                RowStat sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + min(k, K - 1));
+                const int L = len_of(R, b);
+                // (the accept scan saw these row records before it set the sequence's mark; should a load have
+                // overtaken that all the same, ask again)
+                if (k <= L) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
+                if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
                 d.tau = tau_of(R, b);
                 done = &a.p2done[b];
-                skip = k > L;
+                const bool pair = k < L;
+                skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
                 if (!skip) {
-                    const SeqInfo si = ld_cg(a.sinfo + b);
-                    const RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
-                    const RowStat sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + min(k, K - 1));
-                    const bool pair = k < L;
-                    skip = si.n < 0 || (!pair && si.draw_row != L);
-                    if (!skip) {
-                        d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
-                        d.P = row_scale(sp);
-                        if (pair) d.Q = row_scale(sq);
-                        row0 = row_ptr(R, b, k);
-                        if (pair) row1 = row_ptr(R, b, K + 1 + k);
-                    }
+                    d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
+                    d.P = row_scale(sp);
+                    if (pair) d.Q = row_scale(sq);
+                    row0 = row_ptr(R, b, k);
+                    if (pair) row1 = row_ptr(R, b, K + 1 + k);
                 }
             }
             const int n_row = min(left, per_row - s);         // tasks of this run in this row
+            PLOG(24 + (skip ? 1 : 0), b * 100 + r);
             if (skip) {
                 if (done) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" :: "l"(done), "r"(n_row) : "memory");
             } else {
@@ -391,10 +402,9 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
         a.o.accept_len[b] = nn;
         if (a.o.row_status) a.o.row_status[b] = seq_st;
         a.stop[b] = fatal ? -1 : nn;
-        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = 0; si.pad = 0;
-        a.sinfo[b] = si;
-        __threadfence();
-        release_add(&a.adone[b]);
+        // the record's mark makes it (and, through the row records it was computed from, the sequence) ready
+        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = 0; si.pad = 1;
+        st16(a.sinfo + b, si);
     }
 }
 
@@ -716,7 +726,6 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.ticket = reinterpret_cast<int*>(w);
     wa.wait_failed = wa.ticket + 1;
     wa.p1done = reinterpret_cast<int*>(w + wp.off_p1done);
-    wa.adone = reinterpret_cast<int*>(w + wp.off_adone);
     wa.p2done = reinterpret_cast<int*>(w + wp.off_p2done);
     wa.rowcnt = reinterpret_cast<int*>(w + wp.off_rowcnt);
     wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);

@@ -52,7 +52,6 @@ struct WaveArgs {
     int* ticket;          // [1]
     int* wait_failed;     // [1]
     int* p1done;          // [nwaves]
-    int* adone;           // [nwaves]
     int* p2done;          // [nwaves]
     int* rowcnt;          // [B][2K+1] pipelined kernel: softmax partials delivered per row
     P1Part* part;         // [B][2K+1][T]
