@@ -43,6 +43,16 @@ constexpr int PC = WT;                            // consumer threads (8 warps);
 constexpr int PT = PC + 64;                       // + producer warp + publisher warp
 constexpr int PSLICE = kPipeSliceVecs;            // vectors per stage
 constexpr int STAGE_BYTES = PSLICE * 16;
+#ifndef BEBOP_PIPE_LAGD
+#define BEBOP_PIPE_LAGD 0
+#endif
+#ifndef BEBOP_PIPE_NOHINT
+#define BEBOP_PIPE_NOHINT 0
+#endif
+#ifndef BEBOP_PIPE_LAG_MB
+#define BEBOP_PIPE_LAG_MB 0
+#endif
+constexpr size_t kLagBytes = (size_t)BEBOP_PIPE_LAG_MB << 20;   // logits between the first sweep and the second
 constexpr int kPend = 4;                          // runs a producer may set aside
 #ifndef BEBOP_PIPE_BATCH
 #define BEBOP_PIPE_BATCH 2
@@ -106,9 +116,18 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity
     return false;
 }
 // contiguous copy global -> shared of this CTA; 16-byte aligned on both sides, size a multiple of 16
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// `policy`: an L2 eviction policy (first sweep: keep, the second sweep comes back for these lines; second sweep: drop)
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar,
+                                          unsigned long long policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long l2_policy(bool keep) {
+    unsigned long long p;
+    if (BEBOP_PIPE_NOHINT) asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    else if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
 __device__ __forceinline__ void release_add(int* p) {
@@ -147,17 +166,26 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     const int B = R.B;
     const int c0 = NR * T, c2 = (K + 1) * T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
-    // Ticket order: all of P1, then all of P2, then all of D, sequences ascending: the first sequences' accept
-    // scans are long done when the second sweep starts.  Every logit comes from DRAM once per sweep.
-    const int n1 = B * c0, n2 = B * c2;
-    // the run of block-consecutive tasks that starts at ticket t and has at most `want` tasks
+    // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W, then D of sequence
+    // i - W - WD (each where the sequence exists).  With W = B (the default) that is all of P1, then P2 with D
+    // trailing it by WD sequences: two full sweeps, sequences ascending, so that the first sequences' accept scans
+    // are long done when the second sweep starts.  A smaller W pairs the sweeps (the second finds some of its
+    // logits still in L2: the first sweep asks L2 to keep them, the second to drop them) at the price of waiting.
+    const int W = a.lag, WD = a.lag_d;
+    const unsigned long long pol_keep = l2_policy(true), pol_drop = l2_policy(false);
+    auto clampB = [&](int x) { return x < 0 ? 0 : (x > B ? B : x); };
+    auto before = [&](int i) { return c0 * clampB(i) + c2 * clampB(i - W) + clampB(i - W - WD); };   // tickets before block i
+    int blk = 0, f_here = 0, f_next = before(1);      // tickets of this CTA only grow: the block is tracked, not searched
+    // the run of consecutive tasks of one sequence and phase that starts at ticket t, at most `want` tasks;
+    // Run.wv is the sequence, Run.off the offset inside the sequence's block of that phase
     auto decode = [&](int t, int want) {
+        while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
         Run r;
-        r.wv = 0;
-        int room;
-        if (t < n1) { r.ph = 0; r.off = t; room = n1 - t; }
-        else if (t < n1 + n2) { r.ph = 2; r.off = t - n1; room = n1 + n2 - t; }
-        else { r.ph = 3; r.off = t - n1 - n2; room = a.ntickets - t; }
+        int o = t - f_here, room;
+        const int n0 = blk < B ? c0 : 0, n2 = (blk - W >= 0 && blk - W < B) ? c2 : 0;
+        if (o < n0) { r.ph = 0; r.wv = blk; r.off = o; room = n0 - o; }
+        else if (o < n0 + n2) { r.ph = 2; r.wv = blk - W; r.off = o - n0; room = n0 + n2 - o; }
+        else { r.ph = 3; r.wv = blk - W - WD; r.off = 0; room = 1; }
         r.cnt = min(want, room);
         return r;
     };
@@ -175,8 +203,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         if (ph == 3) return wait ? spin_ge(&a.p2done[b], c2) : ld_acquire(&a.p2done[b]) >= c2;
         return true;
     };
-    // first sequence of a run (runs are cut at sequence boundaries for P2 and D, see below)
-    auto run_seq = [&](const Run& r) { return r.ph == 0 ? r.off / c0 : (r.ph == 2 ? r.off / c2 : r.off); };
+    auto run_seq = [&](const Run& r) { return r.wv; };
 #ifdef BEBOP_TRACE
     long long qprev_ = clock64();
 #endif
@@ -198,7 +225,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             if (bleft == 0 && !exhausted) {
                 bt = next; bleft = min(next_cnt, a.ntickets - bt);
                 if (bleft <= 0) { bleft = 0; exhausted = true; }
-                else { next_cnt = bt + bleft >= n1 ? kBatch2 : kBatch; next = atomicAdd(a.ticket, next_cnt); }
+                else { next_cnt = kBatch; next = atomicAdd(a.ticket, next_cnt); }
             }
             if (bleft == 0) {
                 if (npend > 0) continue;
@@ -210,8 +237,6 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             }
             PLOG(20, bt);
             run = decode(bt, bleft);
-            // a P2 or D run stays within one sequence, so that one readiness check covers it
-            if (run.ph == 2) run.cnt = min(run.cnt, c2 - run.off % c2); else if (run.ph == 3) run.cnt = 1;
             bt += run.cnt; bleft -= run.cnt;
             PLOG(21, run_seq(run));
             if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; PLOG(22, run_seq(run)); continue; }
@@ -220,10 +245,10 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         // ---- the tasks of the run
         const int ph = run.ph, wv = 0;
         const int per_row = ph == 0 ? T : (ph == 2 ? T2 : 1), rows = ph == 0 ? NR : (ph == 2 ? K + 1 : 1);
-        int s = run.off % per_row, r = (run.off / per_row) % rows, bb = run.off / (per_row * rows);
+        int s = run.off % per_row, r = (run.off / per_row) % rows;
+        const int b = run.wv;                      // a run stays within one sequence
         int left = run.cnt;
         while (left > 0) {
-            const int b = bb;
             // the row's numbers
             TaskDesc d;
             d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f;
@@ -290,8 +315,9 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                     const uint32_t bytes = (uint32_t)d.nv * 16u;
                     if (row0 && bytes) {
                         mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
-                        bulk_load(data + (size_t)stage * STAGE_BYTES, row0 + (int64_t)d.v0 * 16, bytes, &S.full[stage]);
-                        if (row1) bulk_load(data + (size_t)stage * STAGE_BYTES + STAGE_BYTES / 2, row1 + (int64_t)d.v0 * 16, bytes, &S.full[stage]);
+                        const unsigned long long pol = ph == 0 ? pol_keep : pol_drop;
+                        bulk_load(data + (size_t)stage * STAGE_BYTES, row0 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
+                        if (row1) bulk_load(data + (size_t)stage * STAGE_BYTES + STAGE_BYTES / 2, row1 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
                     } else {
                         mbar_arrive(&S.full[stage]);
                     }
@@ -300,7 +326,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             }
             left -= n_row;
             s = 0;
-            if (++r == rows) { r = 0; ++bb; }
+            ++r;
         }
     }
 }
@@ -740,7 +766,19 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
         const long long total = (long long)a.B * (NR * wp.T + (long long)(a.K + 1) * 2 * wp.T + 1);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
-        wa.lag = wp.lag;
+        // Distance of the second sweep behind the first, in sequences.  The default is the whole batch (two full
+        // sweeps): measured at the headline shape, a second sweep 24 / 48 / 72 / 96 MB of logits behind the first
+        // found a sixth of its lines in L2 at best, and waited for accept scans more than that saved (0.42 / 0.38 /
+        // 0.35 / 0.30 ms against 0.24 ms).  BEBOP_PIPE_LAG_MB > 0 builds the paired order for experiments.
+        long lag = a.B;
+        if (BEBOP_PIPE_LAG_MB > 0) {
+            const size_t seq_bytes = (size_t)NR * a.nvec * 16;
+            lag = (long)(kLagBytes / (seq_bytes ? seq_bytes : 1));
+            if (lag < 4) lag = 4;
+            if (lag > a.B) lag = a.B;
+        }
+        wa.lag = (int)lag;
+        wa.lag_d = (BEBOP_PIPE_LAGD > 0 && BEBOP_PIPE_LAGD < a.B) ? BEBOP_PIPE_LAGD : a.B;   // D tickets: behind P2, or all at the end
     }
     cudaError_t e = cudaMemsetAsync(w, 0, wp.zero_bytes, stream);
     if (e != cudaSuccess) return e;

@@ -59,7 +59,7 @@ struct WaveArgs {
     unsigned long long* dacc;    // [B][2T][2] draw-row mass (2^-58) and sum of squares (2^-40), each << 4 | parts added
     unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
-    int ntickets, lag;
+    int ntickets, lag, lag_d;        // distance (sequences) of P2 behind P1 and of D behind P2
     long long* trace;
     int T, slice_vecs, wave_seqs, nwaves;
 };
