@@ -73,9 +73,6 @@ struct __align__(16) TaskDesc {
     int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from
     float tau;
     RowScale P, Q;
-#ifdef BEBOP_TRACE
-    long long t_issue;
-#endif
 };
 
 struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of one (phase, wave) block from offset off
@@ -90,9 +87,6 @@ struct PipeShared {
     int wi[NST][WW];
     Run pend[kPend];                            // producer: runs set aside
     int logn;                                   // trace builds: events logged
-#ifdef BEBOP_TRACE
-    long long t_empty[NST];
-#endif
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -134,18 +128,6 @@ __device__ __forceinline__ void release_add(int* p) {
     asm volatile("red.release.gpu.global.add.s32 [%0], 1;" :: "l"(p) : "memory");
 }
 
-#ifdef BEBOP_TRACE
-// per wave timeline (ns): [64 + 8*w + i]: 0 first P1 ticket, 1 last row merged, 2 last accept done, 3 first P2 ticket seen,
-// 4 first P2 task published, 5 last P2 partial done, 6 first D ticket seen, 7 last D done
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-__device__ __forceinline__ void tl_min(const WaveArgs& a, int w, int i) { if (a.trace) atomicMin(reinterpret_cast<unsigned long long*>(a.trace) + 64 + 8 * w + i, (unsigned long long)gtime()); }
-__device__ __forceinline__ void tl_max(const WaveArgs& a, int w, int i) { if (a.trace) atomicMax(reinterpret_cast<unsigned long long*>(a.trace) + 64 + 8 * w + i, (unsigned long long)gtime()); }
-#define TL_MIN(w, i) tl_min(a, w, i)
-#define TL_MAX(w, i) tl_max(a, w, i)
-#else
-#define TL_MIN(w, i) do { } while (0)
-#define TL_MAX(w, i) do { } while (0)
-#endif
 
 #ifdef BEBOP_TRACE
 // event log of one CTA: (clock, code * 1e6 + task number)
@@ -204,9 +186,6 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         return true;
     };
     auto run_seq = [&](const Run& r) { return r.wv; };
-#ifdef BEBOP_TRACE
-    long long qprev_ = clock64();
-#endif
     int npend = 0;
     bool exhausted = false;
     int bt = 0, bleft = 0;                         // tickets of the claimed batch not yet turned into runs
@@ -235,12 +214,9 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 mbar_arrive(&S.full[stage]);
                 return;
             }
-            PLOG(20, bt);
             run = decode(bt, bleft);
             bt += run.cnt; bleft -= run.cnt;
-            PLOG(21, run_seq(run));
-            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; PLOG(22, run_seq(run)); continue; }
-            PLOG(23, run_seq(run));
+            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; continue; }
         }
         // ---- the tasks of the run
         const int ph = run.ph, wv = 0;
@@ -287,7 +263,6 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 }
             }
             const int n_row = min(left, per_row - s);         // tasks of this run in this row
-            PLOG(24 + (skip ? 1 : 0), b * 100 + r);
             if (skip) {
                 if (done) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" :: "l"(done), "r"(n_row) : "memory");
             } else {
@@ -295,21 +270,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 for (int i = 0; i < n_row; ++i) {
                     const int stage = it % NST;
                     d.s = s + i; d.v0 = d.s * sv; d.nv = max(min(sv, R.nvec - d.v0), 0);
-#ifdef BEBOP_TRACE
-                    const long long q0_ = clock64();
-#endif
                     if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
-#ifdef BEBOP_TRACE
-                    const long long q1_ = clock64();
-                    d.t_issue = q1_;
-                    if (a.trace && a.trace[4095] != 0) {
-                        unsigned long long* tq = reinterpret_cast<unsigned long long*>(a.trace) + 32 + ph * 8;
-                        atomicAdd(tq + 0, (unsigned long long)(q0_ - qprev_)); atomicAdd(tq + 1, (unsigned long long)(q1_ - q0_)); atomicAdd(tq + 2, 1ull);
-                        if (it >= NST) atomicAdd(tq + 3, (unsigned long long)(q1_ - S.t_empty[stage]));
-                    }
-                    qprev_ = q1_;
-                    if (a.trace && blockIdx.x == 5 && it < 100) { a.trace[2048 + it * 20] = q1_; a.trace[2048 + it * 20 + 17] = ph; }
-#endif
                     S.desc[stage] = d;
                     PLOG(1 + 10 * ph, it);
                     const uint32_t bytes = (uint32_t)d.nv * 16u;
@@ -452,13 +413,20 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
     const TempScale ts = temp_scale(d.tau);
     const int nv = d.nv;
     uint4 raw[NV];
+    if (nv >= (NV - 1) * PC) {                   // the usual case: only a thread's last vector may lie beyond the slice
 #pragma unroll
-    for (int u = 0; u < NV; ++u) {
-        const int v = tid + u * PC;
-        raw[u] = neg_inf_vec<DT>();
-        if (v < nv) raw[u] = lds16(data + (size_t)v * 16);
+        for (int u = 0; u < NV - 1; ++u) raw[u] = lds16(data + (size_t)(tid + u * PC) * 16);
+        raw[NV - 1] = neg_inf_vec<DT>();
+        if (tid + (NV - 1) * PC < nv) raw[NV - 1] = lds16(data + (size_t)(tid + (NV - 1) * PC) * 16);
+    } else {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int v = tid + u * PC;
+            raw[u] = neg_inf_vec<DT>();
+            if (v < nv) raw[u] = lds16(data + (size_t)v * 16);
+        }
     }
-    if ((d.v0 + nv) * VEC > R.V) {
+    if ((d.v0 + nv) * VEC > R.V) {               // the row's last vector is in this slice and is partial
 #pragma unroll
         for (int u = 0; u < NV; ++u) {
             const int gbase = (d.v0 + tid + u * PC) * VEC;
@@ -512,12 +480,21 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
     const bool pair = (d.flags & 1) != 0, draw = (d.flags & 2) != 0;
     const int nv = d.nv;
     const unsigned char* qdata = data + STAGE_BYTES / 2;
+    // Vectors beyond the slice, and the draft row of a bonus task, read as -inf: they give p = q = 0 and add
+    // nothing, so the arithmetic below runs unguarded.
     uint4 rp[NV], rq[NV];
+    if (nv >= (NV - 1) * PC && pair) {           // the usual case: only a thread's last vector may lie beyond the slice
 #pragma unroll
-    for (int u = 0; u < NV; ++u) {
-        const int v = tid + u * PC;
-        rp[u] = neg_inf_vec<DT>(); rq[u] = neg_inf_vec<DT>();
-        if (v < nv) { rp[u] = lds16(data + (size_t)v * 16); if (pair) rq[u] = lds16(qdata + (size_t)v * 16); }
+        for (int u = 0; u < NV - 1; ++u) { rp[u] = lds16(data + (size_t)(tid + u * PC) * 16); rq[u] = lds16(qdata + (size_t)(tid + u * PC) * 16); }
+        rp[NV - 1] = neg_inf_vec<DT>(); rq[NV - 1] = neg_inf_vec<DT>();
+        if (tid + (NV - 1) * PC < nv) { rp[NV - 1] = lds16(data + (size_t)(tid + (NV - 1) * PC) * 16); rq[NV - 1] = lds16(qdata + (size_t)(tid + (NV - 1) * PC) * 16); }
+    } else {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int v = tid + u * PC;
+            rp[u] = neg_inf_vec<DT>(); rq[u] = neg_inf_vec<DT>();
+            if (v < nv) { rp[u] = lds16(data + (size_t)v * 16); if (pair) rq[u] = lds16(qdata + (size_t)v * 16); }
+        }
     }
     const TempScale c = temp_scale(d.tau);
     const RowScale SP = d.P, SQ = d.Q;
@@ -533,27 +510,23 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
     if (!draw) {
 #pragma unroll
         for (int u = 0; u < NV; ++u) {
-            if (tid + u * PC < nv) {
-                float r[8];
+            float r[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                residual_vec<DT, false>(rp[u], rq[u], pair, c, SP, SQ, r, nullptr);
-                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-                if (u & 1) z1 += vs; else z0 += vs;
-            }
+            for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            residual_vec<DT, false>(rp[u], rq[u], c, SP, SQ, r, nullptr);
+            const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+            if (u & 1) z1 += vs; else z0 += vs;
         }
     } else {
 #pragma unroll
         for (int u = 0; u < NV; ++u) {
-            if (tid + u * PC < nv) {
-                float r[8];
+            float r[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                residual_vec<DT, true>(rp[u], rq[u], pair, c, SP, SQ, r, &sqs);
-                const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-                z0 += vs;
-                zd += (double)vs;
-            }
+            for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            residual_vec<DT, true>(rp[u], rq[u], c, SP, SQ, r, &sqs);
+            const float vs = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+            z0 += vs;
+            zd += (double)vs;
         }
     }
     const float z = warp_sum(z0 + z1);
@@ -666,16 +639,10 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     for (int it = 0;; ++it) {
         const int stage = it % NST;
         const uint32_t par = (uint32_t)(it / NST) & 1u;
-#ifdef BEBOP_TRACE
-        const long long c0_ = clock64();
-#endif
         if (!mbar_wait(&S.full[stage], par)) { if (tid == 0) atomicExch(a.wait_failed, 1); break; }
         const TaskDesc d = S.desc[stage];
         if (d.phase < 0) break;
         if (tid == 0) PLOG(2, it);
-#ifdef BEBOP_TRACE
-        const long long c1_ = clock64();
-#endif
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
         if (d.phase == 0) pipe_p1<DT>(a, S, d, sd, stage, it);
         else if (d.phase == 2) pipe_p2<DT>(a, S, d, sd, stage, it);
@@ -686,19 +653,7 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
 
         }
         __syncwarp();
-#ifdef BEBOP_TRACE
-        if (lane == 0) S.t_empty[stage] = clock64();
-#endif
         if (lane == 0) mbar_arrive(&S.empty[stage]);
-#ifdef BEBOP_TRACE
-        if (a.trace && lane == 0 && blockIdx.x == 5 && it < 100) { a.trace[2048 + it * 20 + 1 + (tid >> 5)] = c1_; a.trace[2048 + it * 20 + 9 + (tid >> 5)] = clock64(); }
-        if (a.trace && lane == 0 && a.trace[4095] != 0) {       // per phase and warp-task: cycles waiting for the stage, cycles of the task, count
-            unsigned long long* tq = reinterpret_cast<unsigned long long*>(a.trace) + d.phase * 8;
-            atomicAdd(tq + 0, (unsigned long long)(c1_ - c0_)); atomicAdd(tq + 1, (unsigned long long)(clock64() - c1_));
-            atomicAdd(tq + 2, 1ull);
-            atomicAdd(tq + 3, (unsigned long long)(c1_ - d.t_issue));
-        }
-#endif
     }
 }
 

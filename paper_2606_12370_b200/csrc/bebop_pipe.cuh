@@ -153,20 +153,22 @@ __device__ __forceinline__ RowScale no_row() { RowScale r; r.ef = 0.f; r.inv = 0
 
 // FINE (the rows a token is drawn from): the normaliser enters as two floats, so that its rounding to fp32
 // is not an error common to all tokens of the row; what is left is one rounding per token.
+// A row that is not there (the draft row of a bonus task, vectors beyond the slice) is passed as -inf logits
+// with a zero normaliser: it gives q = 0 without a branch.
 template <int DT, bool FINE>
-__device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, bool pair, const TempScale& c, const RowScale& P,
+__device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, const TempScale& c, const RowScale& P,
                                              const RowScale& Q, float* r, float* sq) {
     constexpr int VEC = Elem<DT>::VEC;
     float fp[VEC], fq[VEC];
     unpack<DT>(rp, fp);
-    if (pair) unpack<DT>(rq, fq);
+    unpack<DT>(rq, fq);
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
         const float ap = exp2_scaled(fp[i], c, P.ef);
-        const float aq = pair ? exp2_scaled(fq[i], c, Q.ef) : 0.f;
+        const float aq = exp2_scaled(fq[i], c, Q.ef);
         // explicit roundings: a contracted p - a*inv would leave rounding dust when the rows are equal
         const float p = FINE ? __fmaf_rn(ap, P.inv_lo, __fmul_rn(ap, P.inv)) : __fmul_rn(ap, P.inv);
-        const float q = pair ? (FINE ? __fmaf_rn(aq, Q.inv_lo, __fmul_rn(aq, Q.inv)) : __fmul_rn(aq, Q.inv)) : 0.f;
+        const float q = FINE ? __fmaf_rn(aq, Q.inv_lo, __fmul_rn(aq, Q.inv)) : __fmul_rn(aq, Q.inv);
         r[i] = fmaxf(p - q, 0.f);
         if (sq) { *sq = fmaf(p, p, *sq); *sq = fmaf(q, q, *sq); }
     }
@@ -254,7 +256,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b,
             float r[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) r[i] = 0.f;
-            residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
+            residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
             vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
         }
         BEBOP_CTA_SYNC();
@@ -286,7 +288,7 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b,
                     float r[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                    residual_vec<DT, true>(rp, rq, pair, c, SP, SQ, r, nullptr);
+                    residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
                     double Cw = C;
 #pragma unroll
                     for (int i = 0; i < VEC; ++i) {
