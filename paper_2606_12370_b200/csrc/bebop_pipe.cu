@@ -71,7 +71,8 @@ struct __align__(16) TaskDesc {
     int wave, b, r;   // r: row (P1) or draft position (P2)
     int s, v0, nv;    // slice, its first vector, its vectors
     int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from
-    float tau;
+    float tau;        // temperature, and c = log2(e) / tau computed once per row
+    float c;
     RowScale P, Q;
 };
 
@@ -227,7 +228,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         while (left > 0) {
             // the row's numbers
             TaskDesc d;
-            d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f;
+            d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f; d.c = 0.f;
             d.P = no_row(); d.Q = no_row();
             const char* row0 = nullptr; const char* row1 = nullptr;
             bool skip = false;
@@ -236,7 +237,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 const int L = len_of(R, b);
                 const bool is_target = r <= K;
                 const int k = is_target ? r : r - (K + 1);
-                d.tau = tau_of(R, b);
+                d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
                 skip = is_target ? k > L : k >= L;
                 row0 = row_ptr(R, b, r);
             } else if (ph == 2) {
@@ -250,7 +251,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 // overtaken that all the same, ask again)
                 if (k <= L) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
-                d.tau = tau_of(R, b);
+                d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
                 done = &a.p2done[b];
                 const bool pair = k < L;
                 skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
@@ -410,7 +411,7 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const TempScale ts = temp_scale(d.tau);
+    TempScale ts; ts.hi = d.c;
     const int nv = d.nv;
     uint4 raw[NV];
     if (nv >= (NV - 1) * PC) {                   // the usual case: only a thread's last vector may lie beyond the slice
@@ -496,7 +497,7 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
             if (v < nv) { rp[u] = lds16(data + (size_t)v * 16); if (pair) rq[u] = lds16(qdata + (size_t)v * 16); }
         }
     }
-    const TempScale c = temp_scale(d.tau);
+    TempScale c; c.hi = d.c;
     const RowScale SP = d.P, SQ = d.Q;
     if ((d.v0 + nv) * VEC > R.V) {
 #pragma unroll
