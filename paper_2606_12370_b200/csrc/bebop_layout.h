@@ -8,7 +8,7 @@ namespace bebop {
 
 // Workspace of the pipelined kernel and of the fp64 re-draw kernels.
 #ifndef BEBOP_PIPE_SLICE_VECS
-#define BEBOP_PIPE_SLICE_VECS 1536
+#define BEBOP_PIPE_SLICE_VECS 2048
 #endif
 constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
 struct WavePlan {

@@ -32,7 +32,7 @@ namespace bebop {
 namespace {
 
 #ifndef BEBOP_PIPE_STAGES
-#define BEBOP_PIPE_STAGES 3
+#define BEBOP_PIPE_STAGES 2
 #endif
 #ifndef BEBOP_PIPE_CTAS
 #define BEBOP_PIPE_CTAS 3
