@@ -243,7 +243,7 @@ def run_ours(args):
     kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
     kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = 6 if args.path == 1 else 4      # main kernel, flag, 2 fp64 re-draw kernels | 6 general kernels
+    launches_per_call = 6 if args.path == 1 else 3      # main kernel, 2 fp64 re-draw kernels | 6 general kernels
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))

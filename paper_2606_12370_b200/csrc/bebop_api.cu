@@ -188,7 +188,7 @@ void bebop_debug_set_timing_events(void* start, void* stop) { wave_set_events(st
 
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
     if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;
-    return make_plan(B, K, V, (int)dt).off_fb;
+    return make_plan(B, K, V, (int)dt).off_wave + kFbCountOffset;
 }
 
 const char* bebop_status_string(bebop_status_t status) {

@@ -11,6 +11,13 @@ namespace bebop {
 #define BEBOP_PIPE_SLICE_VECS 2048
 #endif
 constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
+// A sequence whose draw goes to the fp64 re-draw: all the re-draw kernels need to find its rows.
+struct alignas(16) FbRec {
+    int b;                              // sequence
+    int kp;                             // 2 * draw row + (1 if the row is a residual of a target / draft pair)
+    int ep, eq;                         // reference exponents of the target row and of the draft row
+};
+constexpr size_t kFbCountOffset = 128;   // int: sequences listed for the fp64 re-draw, inside the zeroed head of the workspace
 struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
     int wave_seqs, nwaves; // sequences per wave, waves
@@ -33,7 +40,7 @@ struct Plan {
     size_t off_dstats;  // double2[B][2][nsplit_d]       (m, S) partials, fp64
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
-    size_t off_fb;      // int [1 + B]: count and list of sequences whose draw goes to fp64
+    size_t off_fb;      // 16-byte records [B]: the sequences whose draw goes to fp64
     size_t off_wave;    // workspace of the pipelined kernel
     size_t total;
 };
@@ -53,7 +60,7 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.wave_seqs = (int)ws;
     w.nwaves = (B + w.wave_seqs - 1) / w.wave_seqs;
     w.lag = 2;
-    size_t o = 256;                                           // ticket, wait flag
+    size_t o = 256;                                           // ticket, wait flag; at kFbCountOffset the re-draw count
     w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per sequence: rows merged
     w.off_adone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
@@ -98,7 +105,7 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dstats = o; o = align256(o + sizeof(double) * 2 * (size_t)B * 2 * nsd);
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
-    p.off_fb = o;     o = align256(o + sizeof(int) * (size_t)(B + 64));
+    p.off_fb = o;     o = align256(o + 16 * (size_t)B);
     {
         p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
     }

@@ -702,9 +702,9 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     WaveArgs wa;
     wa.r = a; wa.draft_tokens = draft_tokens; wa.u_accept = u_accept; wa.u_final = u_final; wa.o = o;
     wa.stop = reinterpret_cast<int*>(ws + p.off_stop);
-    wa.fb_count = reinterpret_cast<int*>(ws + p.off_fb);
-    wa.fb_list = wa.fb_count + 16;
     char* w = ws + p.off_wave;
+    wa.fb_count = reinterpret_cast<int*>(w + kFbCountOffset);
+    wa.fb_list = reinterpret_cast<FbRec*>(ws + p.off_fb);
     wa.ticket = reinterpret_cast<int*>(w);
     wa.wait_failed = wa.ticket + 1;
     wa.p1done = reinterpret_cast<int*>(w + wp.off_p1done);
@@ -738,8 +738,6 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     }
     cudaError_t e = cudaMemsetAsync(w, 0, wp.zero_bytes, stream);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(wa.fb_count, 0, sizeof(int), stream);
-    if (e != cudaSuccess) return e;
     const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
     if (g_ev_start) cudaEventRecord(g_ev_start, stream);
     if (a.dt == 0) k_pipe<0><<<grid, PT, kPipeSmem, stream>>>(wa);
@@ -747,11 +745,8 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     e = cudaGetLastError();
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;
-    wave_flag_launch(wa.wait_failed, o.row_status, a.B, stream);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     *launched = true;
-    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, w, wp, stream);
+    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, wa.wait_failed, w, wp, stream);
 }
 
 }  // namespace bebop

@@ -46,8 +46,8 @@ struct WaveArgs {
     const float* u_final;
     VerifyOut o;
     int* stop;
-    int* fb_count;
-    int* fb_list;
+    int* fb_count;        // [1] sequences listed for the fp64 re-draw (zeroed with the workspace)
+    FbRec* fb_list;       // [B]
     // workspace
     int* ticket;          // [1]
     int* wait_failed;     // [1]
@@ -315,7 +315,13 @@ __device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b,
         int y = -1, cnt = 0;
         for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
         if (cnt == 1 && y >= 0) a.o.out_tokens[(int64_t)b * (K + 1) + k] = y;
-        else { int idx = atomicAdd(a.fb_count, 1); a.fb_list[idx] = b; }
+        else {
+            FbRec rec;
+            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0);
+            rec.ep = ld_cg(a.rstat + (int64_t)b * NR + k).e;
+            rec.eq = pair ? ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k).e : 0;
+            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
+        }
     }
 }
 

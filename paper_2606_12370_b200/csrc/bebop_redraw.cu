@@ -9,9 +9,9 @@ namespace {
 
 // ------------------------------------------------------------------ fp64 re-draw of the listed sequences
 // Two small kernels behind the pipelined kernel, for the few sequences whose fast draw did not clear its
-// error bound.  Every row is cut into XT = 4T quarter slices; CTA (s, y) takes quarter slice s of the
-// listed sequences y, y + gridDim.y, ...  Everything is evaluated in double around the row exponents
-// that phase A left (any common reference cancels in p = a / sum a).
+// error bound.  Every row is cut into XT = 4T quarter slices; the work items (listed sequence, quarter
+// slice) are dealt round-robin to a fixed grid.  Everything is evaluated in double around the row
+// exponents that phase A left (any common reference cancels in p = a / sum a).
 //   k_redraw_sum   exact normalisers: sum of exponentials of each quarter slice of the draw rows;
 //   k_redraw_mass  residual mass of each quarter slice, one sum per warp (warp w owns the contiguous
 //                  vectors [w*cw, (w+1)*cw)); the CTA that completes a sequence picks its token at
@@ -22,14 +22,36 @@ struct RedrawArgs {
     const float* u_final;
     VerifyOut o;
     const int* fb_count;     // listed sequences
-    const int* fb_list;
-    const SeqInfo* sinfo;
-    const RowStat* rstat;
+    const FbRec* fb_list;
+    const int* wait_failed;  // set by a device-side wait of the main kernel that gave up
     double2* xsum;           // [B][XT] sums of exponentials (target row, draft row) per quarter slice
     double* xmass;           // [B][XT][WW] residual mass per quarter slice and warp chunk
     int* xdone;              // [B] per listed sequence: mass tasks finished
     int T, slice_vecs;
 };
+
+// 2^t in double for t <= about 0: t = n/64 + f with |f| <= 1/128, 2^t = 2^(n >> 6) * tab[n & 63] * 2^f,
+// 2^f by its series to the fifth power (the next term is below 4e-17 of the result).  About a dozen
+// double-precision instructions, a third of the library routine; the result is within 2 ulp.
+// `tab` holds 2^(j/64), j = 0..63, in shared memory.  Arguments below -1000 (and -inf) give 0.
+constexpr int XTAB = 64;
+__device__ __forceinline__ void x_exp2_table(double* tab) {
+    if (threadIdx.x < XTAB) tab[threadIdx.x] = exp2((double)threadIdx.x * (1.0 / XTAB));
+}
+__device__ __forceinline__ double x_exp2(double t, const double* tab) {
+    if (!(t > -1000.0)) return 0.0;
+    const double magic = 6755399441055744.0;                 // 1.5 * 2^52: adding it rounds to an integer
+    const double tm = fma(t, (double)XTAB, magic);
+    const int n = __double2loint(tm);
+    const double f = fma(tm - magic, -1.0 / XTAB, t);         // exact
+    double p = fma(f, 0.0013333558146428443, 0.009618129107628477);     // ln2^5/120, ln2^4/24
+    p = fma(f, p, 0.05550410866482158);                                 // ln2^3/6
+    p = fma(f, p, 0.2402265069591007);                                  // ln2^2/2
+    p = fma(f, p, 0.6931471805599453);                                  // ln2
+    const double s = tab[n & (XTAB - 1)];
+    const double r = fma(s * f, p, s);
+    return __hiloint2double(__double2hiint(r) + ((n >> 6) << 20), __double2loint(r));
+}
 
 struct XRow {
     const char* prow; const char* qrow;
@@ -37,30 +59,28 @@ struct XRow {
     int b, k;
     bool pair;
 };
-__device__ __forceinline__ double x_resid(const XRow& d, float zp, float zq) {
+__device__ __forceinline__ double x_resid(const XRow& d, float zp, float zq, const double* tab) {
     // explicit roundings: a contracted p * ip - q would leave rounding dust when p == q
-    const double p = __dmul_rn(exp2(fma((double)zp, d.c, -d.ep)), d.ip);
+    const double p = __dmul_rn(x_exp2(fma((double)zp, d.c, -d.ep), tab), d.ip);
     if (!d.pair) return p;
-    const double q = __dmul_rn(exp2(fma((double)zq, d.c, -d.eq)), d.iq);
+    const double q = __dmul_rn(x_exp2(fma((double)zq, d.c, -d.eq), tab), d.iq);
     const double df = p - q;
     return df > 0.0 ? df : 0.0;
 }
-__device__ __forceinline__ bool x_row(const RedrawArgs& a, int slot, XRow* d) {
+__device__ __forceinline__ void x_row(const RedrawArgs& a, int slot, XRow* d) {
     const RowArgs& R = a.r;
-    const int K = R.K, NR = 2 * K + 1;
-    const int b = a.fb_list[slot];
-    const SeqInfo si = a.sinfo[b];
-    d->b = b; d->k = si.draw_row;
-    if (si.draw_row < 0) return false;
-    d->pair = si.draw_row < len_of(R, b);
-    d->prow = row_ptr(R, b, si.draw_row);
-    d->qrow = d->pair ? row_ptr(R, b, K + 1 + si.draw_row) : d->prow;
+    const FbRec rec = a.fb_list[slot];
+    const int b = rec.b, k = rec.kp >> 1;
+    d->b = b; d->k = k;
+    d->pair = rec.kp & 1;
+    d->prow = row_ptr(R, b, k);
+    d->qrow = d->pair ? row_ptr(R, b, R.K + 1 + k) : d->prow;
     d->c = 1.4426950408889634 / (double)tau_of(R, b);
-    d->ep = (double)a.rstat[(int64_t)b * NR + si.draw_row].e;
-    d->eq = d->pair ? (double)a.rstat[(int64_t)b * NR + K + 1 + si.draw_row].e : 0.0;
+    d->ep = (double)rec.ep;
+    d->eq = (double)rec.eq;
     d->ip = 1.0; d->iq = 1.0;
-    return true;
 }
+constexpr int kRedrawGrid = 148 * 4;
 constexpr int XNU = 2;     // vectors per thread and row in a quarter slice (at most 512 vectors)
 
 // this thread's vectors of quarter slice s: warp chunk [warp*cw, warp*cw + cw), lanes interleaved
@@ -88,11 +108,20 @@ template <int DT>
 __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
     constexpr int VEC = Elem<DT>::VEC;
     __shared__ double sh[2][WW];
+    __shared__ double tab[XTAB];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int XT = 4 * a.T, s = blockIdx.x, count = *a.fb_count;
-    for (int slot = blockIdx.y; slot < count; slot += gridDim.y) {
+    const int XT = 4 * a.T, items = *a.fb_count * XT;
+    // a wait of the main kernel that gave up: every row's status says so
+    if (a.o.row_status && *a.wait_failed) {
+        for (int b = blockIdx.x * WT + tid; b < a.r.B; b += gridDim.x * WT) a.o.row_status[b] |= ST_WAIT;
+    }
+    if ((int)blockIdx.x >= items) return;
+    x_exp2_table(tab);
+    __syncthreads();
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int slot = item / XT, s = item - slot * XT;
         XRow d;
-        if (!x_row(a, slot, &d)) continue;
+        x_row(a, slot, &d);
         float fp[XNU][VEC], fq[XNU][VEC];
         x_load<DT>(a, d, s, fp, fq);
         double sa = 0.0, sb = 0.0;
@@ -100,8 +129,8 @@ __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
         for (int u = 0; u < XNU; ++u) {
 #pragma unroll
             for (int i = 0; i < VEC; ++i) {
-                sa += exp2(fma((double)fp[u][i], d.c, -d.ep));
-                if (d.pair) sb += exp2(fma((double)fq[u][i], d.c, -d.eq));
+                sa += x_exp2(fma((double)fp[u][i], d.c, -d.ep), tab);
+                if (d.pair) sb += x_exp2(fma((double)fq[u][i], d.c, -d.eq), tab);
             }
         }
         sa = warp_sum(sa); sb = warp_sum(sb);
@@ -146,18 +175,24 @@ template <int DT>
 __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
     constexpr int VEC = Elem<DT>::VEC;
     __shared__ PickShared S;
+    __shared__ double tab[XTAB];
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = R.K, XT = 4 * a.T, s = blockIdx.x, count = *a.fb_count;
+    const int K = R.K, XT = 4 * a.T, items = *a.fb_count * XT;
     const int qv = a.slice_vecs >> 2, cw = (qv + WW - 1) / WW;
-    for (int slot = blockIdx.y; slot < count; slot += gridDim.y) {
+    if ((int)blockIdx.x >= items) return;
+    x_exp2_table(tab);
+    __syncthreads();
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int slot = item / XT, s = item - slot * XT;
         XRow d;
-        if (!x_row(a, slot, &d)) continue;
+        x_row(a, slot, &d);
         const int b = d.b;
-        // exact normalisers: quarter-slice sums in slice order (the same order in every CTA)
+        // exact normalisers: every warp adds the quarter-slice sums in the same order (lane t takes sums t,
+        // t + 32, ...; the butterfly leaves the same bits in every lane), so every CTA gets the same value
         double Sa = 0.0, Sb = 0.0;
-#pragma unroll 8
-        for (int t = 0; t < XT; ++t) { const double2 x = a.xsum[(int64_t)b * XT + t]; Sa += x.x; Sb += x.y; }
+        for (int t = lane; t < XT; t += 32) { const double2 x = a.xsum[(int64_t)b * XT + t]; Sa += x.x; Sb += x.y; }
+        Sa = warp_sum(Sa); Sb = warp_sum(Sb);
         d.ip = 1.0 / Sa; d.iq = d.pair ? 1.0 / Sb : 0.0;
         if (d.pair) {     // a bonus row needs no mass pass: its masses are sums of exponentials over Sa
             float fp[XNU][VEC], fq[XNU][VEC];
@@ -166,7 +201,7 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
 #pragma unroll
             for (int u = 0; u < XNU; ++u) {
 #pragma unroll
-                for (int i = 0; i < VEC; ++i) m += x_resid(d, fp[u][i], fq[u][i]);
+                for (int i = 0; i < VEC; ++i) m += x_resid(d, fp[u][i], fq[u][i], tab);
             }
             m = warp_sum(m);
             if (lane == 0) a.xmass[((int64_t)b * XT + s) * WW + warp] = m;
@@ -221,7 +256,7 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
                     float f[VEC];
                     load_vec<DT>(d.prow, p0 + vl, R.V, f);
 #pragma unroll
-                    for (int i = 0; i < VEC; ++i) wm += x_resid(d, f[i], 0.f);
+                    for (int i = 0; i < VEC; ++i) wm += x_resid(d, f[i], 0.f, tab);
                 }
             }
             wm = warp_sum(wm);
@@ -248,7 +283,7 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
             if (i < per && v < e1) {
                 const float zp = load_one<DT>(d.prow, v);
                 const float zq = d.pair ? load_one<DT>(d.qrow, v) : 0.f;
-                r[i] = x_resid(d, zp, zq);
+                r[i] = x_resid(d, zp, zq, tab);
                 mine += r[i];
             }
         }
@@ -282,35 +317,28 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
 
 }  // namespace
 
-__global__ void k_wait_flag(const int* __restrict__ wait_failed, int32_t* row_status, int B) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B && *wait_failed && row_status) row_status[b] |= ST_WAIT;
-}
-
 long long* g_wave_trace = nullptr;
 void wave_set_trace(long long* p) { g_wave_trace = p; }
 cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 void wave_set_events(cudaEvent_t start, cudaEvent_t stop) { g_ev_start = start; g_ev_stop = stop; }
 
-void wave_flag_launch(const int* wait_failed, int32_t* row_status, int B, cudaStream_t stream) {
-    k_wait_flag<<<(B + 255) / 256, 256, 0, stream>>>(wait_failed, row_status, B);
-}
-
 // fp64 re-draw of the listed sequences (usually a few per cent of the batch; the count stays on the device)
 cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const int* fb_count,
-                          const int* fb_list, char* w, const WavePlan& wp, cudaStream_t stream) {
+                          const FbRec* fb_list, const int* wait_failed, char* w, const WavePlan& wp,
+                          cudaStream_t stream) {
     RedrawArgs ra;
     ra.r = a; ra.u_final = u_final; ra.o = o;
-    ra.fb_count = fb_count; ra.fb_list = fb_list;
-    ra.sinfo = reinterpret_cast<const SeqInfo*>(w + wp.off_sinfo);
-    ra.rstat = reinterpret_cast<const RowStat*>(w + wp.off_rstat);
+    ra.fb_count = fb_count; ra.fb_list = fb_list; ra.wait_failed = wait_failed;
     ra.xsum = reinterpret_cast<double2*>(w + wp.off_xsum);
     ra.xmass = reinterpret_cast<double*>(w + wp.off_xmass);
     ra.xdone = reinterpret_cast<int*>(w + wp.off_xdone);
     ra.T = wp.T; ra.slice_vecs = wp.slice_vecs;
-    const dim3 rgrid(4 * wp.T, a.B < 32 ? a.B : 32);
-    if (a.dt == 0) { k_redraw_sum<0><<<rgrid, WT, 0, stream>>>(ra); k_redraw_mass<0><<<rgrid, WT, 0, stream>>>(ra); }
-    else { k_redraw_sum<1><<<rgrid, WT, 0, stream>>>(ra); k_redraw_mass<1><<<rgrid, WT, 0, stream>>>(ra); }
+    // the count of listed sequences stays on the device: a fixed grid, four CTAs per SM, takes the work
+    // items round-robin (a CTA without an item returns at once)
+    const long items_max = (long)a.B * 4 * wp.T;
+    const int grid = (int)(items_max < kRedrawGrid ? items_max : kRedrawGrid);
+    if (a.dt == 0) { k_redraw_sum<0><<<grid, WT, 0, stream>>>(ra); k_redraw_mass<0><<<grid, WT, 0, stream>>>(ra); }
+    else { k_redraw_sum<1><<<grid, WT, 0, stream>>>(ra); k_redraw_mass<1><<<grid, WT, 0, stream>>>(ra); }
     return cudaGetLastError();
 }
 
