@@ -49,13 +49,14 @@ def ncu_traffic(kernel):
     return None
 
 
-def roofline(alg_bytes, kern_ms, peak, peak_kind, headline, kernel):
+def roofline(alg_bytes, kern_ms, peak, peak_kind, headline, kernel, timed_launches):
     """HBM roofline of the dominant kernel: algorithmic bytes of one launch over its CUDA-event
     duration measured inside the timed region."""
     gbs = alg_bytes / (kern_ms * 1e-3) / 1e9
     return {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
             "traffic": ncu_traffic(kernel) if headline else None, "peak_kind": "of " + peak_kind,
-            "kernel": kernel, "kernel_ms": kern_ms, "algorithmic_bytes_per_launch": alg_bytes,
+            "kernel": kernel, "kernel_ms": kern_ms, "kernel_launches_timed": timed_launches,
+            "algorithmic_bytes_per_launch": alg_bytes,
             "pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS}
 
 
@@ -220,8 +221,9 @@ def run_ours(args):
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # events around the dominant kernel (k_pipe) inside the timed region: the library records
-    # them on the launching stream; at most 256 steps carry a pair
-    stride = max(1, steps // 256)
+    # them on the launching stream.  Every fourth step at most, and at most 32 steps, carry a pair: an
+    # event between the main kernel and its dependent kernels costs that step about 5 us
+    stride = max(4, (steps + 31) // 32)
     pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
              for _ in range((steps + stride - 1) // stride)]
     for a_, b_ in pairs:            # a torch event owns a CUDA event only after its first record
@@ -297,7 +299,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3},
             "gpu_launches": steps * launches_per_call,
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,
-            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256, KERNEL_OF_PATH.get(args.path, "general kernels")),
+            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256, KERNEL_OF_PATH.get(args.path, "general kernels"), len(pairs)),
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle

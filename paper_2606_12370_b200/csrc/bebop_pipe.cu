@@ -29,6 +29,25 @@
 
 namespace bebop {
 
+#ifdef BEBOP_TRACE
+// timeline of the kernel: [2i] earliest, [2i+1] latest global-timer stamp of event i over all CTAs
+__device__ unsigned long long g_pipe_trace[32];
+__device__ __forceinline__ void pt_log(int i) {
+    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(&g_pipe_trace[2 * i], t); atomicMax(&g_pipe_trace[2 * i + 1], t);
+}
+#define PTLOG(i) pt_log(i)
+extern "C" void bebop_debug_pipe_trace(unsigned long long* host32, int reset) {
+    if (reset) {
+        unsigned long long init[32];
+        for (int i = 0; i < 16; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
+        cudaMemcpyToSymbol(g_pipe_trace, init, sizeof(init));
+    } else cudaMemcpyFromSymbol(host32, g_pipe_trace, 32 * sizeof(unsigned long long));
+}
+#else
+#define PTLOG(i) do { } while (0)
+#endif
+
 namespace {
 
 #ifndef BEBOP_PIPE_STAGES
@@ -43,9 +62,6 @@ constexpr int PC = WT;                            // consumer threads (8 warps);
 constexpr int PT = PC + 64;                       // + producer warp + publisher warp
 constexpr int PSLICE = kPipeSliceVecs;            // vectors per stage
 constexpr int STAGE_BYTES = PSLICE * 16;
-#ifndef BEBOP_PIPE_LAGD
-#define BEBOP_PIPE_LAGD 0
-#endif
 #ifndef BEBOP_PIPE_NOHINT
 #define BEBOP_PIPE_NOHINT 0
 #endif
@@ -70,11 +86,25 @@ struct __align__(16) TaskDesc {
     int phase;        // 0 P1, 1 A, 2 P2, 3 D, -1: no more tasks
     int wave, b, r;   // r: row (P1) or draft position (P2)
     int s, v0, nv;    // slice, its first vector, its vectors
-    int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from
+    int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from,
+                      // bit 2 (D): no half slice owns the target, the draw goes to the fp64 re-draw
     float tau;        // temperature, and c = log2(e) / tau computed once per row
     float c;
     RowScale P, Q;
+    int need;         // P2: partials the sequence's second sweep delivers in all (the last one starts the draw's set-up)
+    float bound;      // D: the error bound the draw must clear,
+    double tt, base;  //    the target of the inverse CDF and the mass before the half slice in the stage
 };
+
+// A draw the publisher warp hands to the producer of its CTA: sequence, draw row, the half slice that owns the
+// target of the inverse CDF, and the numbers the task needs.
+struct DrawTask {
+    double tt, base;
+    float bound, c;
+    int b, k, owner, pair;
+    RowScale P, Q;
+};
+constexpr int kMbox = 8;                     // mailbox entries: more than the tasks a CTA can have unpublished
 
 struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of one (phase, wave) block from offset off
 
@@ -87,6 +117,12 @@ struct PipeShared {
     double wd[NST][WW];
     int wi[NST][WW];
     Run pend[kPend];                            // producer: runs set aside
+    DrawTask mbox[kMbox];                       // publisher -> producer: draws to stage
+    int mb_tail, mb_head;                       // entries written (publisher) and taken (producer)
+    int pub_count;                              // streaming tasks the publisher has dealt with
+    float vsum[PSLICE / 2];                     // D: residual mass per vector of the half slice
+    double d1_tot[2 * MAX_SLICES];              // publisher: half-slice masses and sums of squares of a sequence
+    float d1_sq[2 * MAX_SLICES];
     int logn;                                   // trace builds: events logged
 };
 
@@ -138,10 +174,12 @@ __device__ __forceinline__ void release_add(int* p) {
 #endif
 
 // ------------------------------------------------------------------ producer
-// One thread.  Tickets are claimed kBatch at a time; consecutive tickets of one (phase, wave) block are
+// One thread.  Tickets are claimed kBatch at a time; consecutive tickets of one (phase, sequence) block are
 // consecutive slices of a row, then the next row, then the next sequence, so a batch decodes once and
 // then steps, and the per-row numbers (length, temperature, normalisers, row addresses) are fetched
-// once per row.  Returns when the stop description has been handed to the consumers.
+// once per row.  Draw tasks have no tickets: the publisher warp of this CTA leaves one in the CTA's mailbox
+// when it has delivered the last partial of a sequence's second sweep, and the producer stages it ahead of
+// the next ticket.  Returns when the stop description has been handed to the consumers.
 template <int DT>
 __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsigned char* data) {
     const RowArgs& R = a.r;
@@ -149,15 +187,15 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     const int B = R.B;
     const int c0 = NR * T, c2 = (K + 1) * T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
-    // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W, then D of sequence
-    // i - W - WD (each where the sequence exists).  With W = B (the default) that is all of P1, then P2 with D
-    // trailing it by WD sequences: two full sweeps, sequences ascending, so that the first sequences' accept scans
-    // are long done when the second sweep starts.  A smaller W pairs the sweeps (the second finds some of its
-    // logits still in L2: the first sweep asks L2 to keep them, the second to drop them) at the price of waiting.
-    const int W = a.lag, WD = a.lag_d;
+    // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
+    // exists).  With W = B (the default) that is all of P1, then all of P2: two full sweeps, sequences ascending,
+    // so that the first sequences' accept scans are long done when the second sweep starts.  A smaller W pairs
+    // the sweeps (the second finds some of its logits still in L2: the first sweep asks L2 to keep them, the
+    // second to drop them) at the price of waiting.
+    const int W = a.lag;
     const unsigned long long pol_keep = l2_policy(true), pol_drop = l2_policy(false);
     auto clampB = [&](int x) { return x < 0 ? 0 : (x > B ? B : x); };
-    auto before = [&](int i) { return c0 * clampB(i) + c2 * clampB(i - W) + clampB(i - W - WD); };   // tickets before block i
+    auto before = [&](int i) { return c0 * clampB(i) + c2 * clampB(i - W); };   // tickets before block i
     int blk = 0, f_here = 0, f_next = before(1);      // tickets of this CTA only grow: the block is tracked, not searched
     // the run of consecutive tasks of one sequence and phase that starts at ticket t, at most `want` tasks;
     // Run.wv is the sequence, Run.off the offset inside the sequence's block of that phase
@@ -165,16 +203,15 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
         Run r;
         int o = t - f_here, room;
-        const int n0 = blk < B ? c0 : 0, n2 = (blk - W >= 0 && blk - W < B) ? c2 : 0;
+        const int n0 = blk < B ? c0 : 0;
         if (o < n0) { r.ph = 0; r.wv = blk; r.off = o; room = n0 - o; }
-        else if (o < n0 + n2) { r.ph = 2; r.wv = blk - W; r.off = o - n0; room = n0 + n2 - o; }
-        else { r.ph = 3; r.wv = blk - W - WD; r.off = 0; room = 1; }
+        else { r.ph = 2; r.wv = blk - W; r.off = o - n0; room = n0 + c2 - o; }
         r.cnt = min(want, room);
         return r;
     };
-    // Is sequence b ready for the phase?  P2 needs its accept scan, D all of its P2 partials.  A run that is
-    // not ready is set aside (up to kPend of them) while later tickets go ahead; the oldest one is looked at
-    // again before every new run and waited for only when the shelf is full or no tickets are left.
+    // Is sequence b ready for the phase?  P2 needs its accept scan.  A run that is not ready is set aside (up to
+    // kPend of them) while later tickets go ahead; the oldest one is looked at again before every new run and
+    // waited for only when the shelf is full or no tickets are left.
     // the sequence's record of the accept scan, valid once its mark is set (waits, bounded, if asked to)
     auto seq_info = [&](int b, bool wait) {
         SeqInfo si = ld_cg(a.sinfo + b);
@@ -183,32 +220,70 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     };
     auto ready = [&](int ph, int b, bool wait) {
         if (ph == 2) return seq_info(b, wait).pad != 0;
-        if (ph == 3) return wait ? spin_ge(&a.p2done[b], c2) : ld_acquire(&a.p2done[b]) >= c2;
         return true;
     };
-    auto run_seq = [&](const Run& r) { return r.wv; };
+    int it = 0, n_stream = 0, mb_head = 0;
+    // hand one task to the consumers: its description, and its logits on their way into the stage
+    auto issue = [&](const TaskDesc& d, const char* row0, const char* row1, unsigned long long pol) {
+        const int stage = it % NST;
+        if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
+        S.desc[stage] = d;
+        PLOG(1 + 10 * d.phase, it);
+        const uint32_t bytes = (uint32_t)d.nv * 16u;
+        if (row0 && bytes) {
+            mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
+            bulk_load(data + (size_t)stage * STAGE_BYTES, row0 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
+            if (row1) bulk_load(data + (size_t)stage * STAGE_BYTES + STAGE_BYTES / 2, row1 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
+        } else {
+            mbar_arrive(&S.full[stage]);
+        }
+        ++it;
+    };
+    // the draw tasks the publisher left in the mailbox: the half slice that owns the target, staged like a P2 task
+    auto drain = [&]() {
+        while (mb_head != *(volatile int*)&S.mb_tail) {
+            const DrawTask t = S.mbox[mb_head % kMbox];
+            ++mb_head;
+            *(volatile int*)&S.mb_head = mb_head;
+            TaskDesc d;
+            d.phase = 3; d.wave = 0; d.b = t.b; d.r = t.k; d.s = t.owner; d.flags = (t.pair ? 1 : 0) | 2;
+            d.v0 = t.owner * sv2; d.nv = max(min(sv2, R.nvec - d.v0), 0);
+            d.tau = 1.f; d.c = t.c; d.P = t.P; d.Q = t.Q; d.need = 0;
+            d.bound = t.bound; d.tt = t.tt; d.base = t.base;
+            issue(d, row_ptr(R, t.b, t.k), t.pair ? row_ptr(R, t.b, K + 1 + t.k) : nullptr, pol_drop);
+        }
+    };
     int npend = 0;
     bool exhausted = false;
     int bt = 0, bleft = 0;                         // tickets of the claimed batch not yet turned into runs
-    int next_cnt = kBatch;                         // tickets of the claim in flight (more at a time in the second sweep)
+    int next_cnt = kBatch;                         // tickets of the claim in flight
     int next = atomicAdd(a.ticket, next_cnt);
-    int it = 0;
     for (;;) {
+        drain();
         // ---- next run
         Run run;
-        if (npend > 0 && (ready(S.pend[0].ph, run_seq(S.pend[0]), false) || npend == kPend || (exhausted && bleft == 0))) {
+        if (npend > 0 && (ready(S.pend[0].ph, S.pend[0].wv, false) || npend == kPend || (exhausted && bleft == 0))) {
             run = S.pend[0];
-            if (!ready(run.ph, run_seq(run), true)) atomicExch(a.wait_failed, 1);
+            if (!ready(run.ph, run.wv, true)) atomicExch(a.wait_failed, 1);
             --npend;
             for (int i = 0; i < npend; ++i) S.pend[i] = S.pend[i + 1];
         } else {
             if (bleft == 0 && !exhausted) {
                 bt = next; bleft = min(next_cnt, a.ntickets - bt);
-                if (bleft <= 0) { bleft = 0; exhausted = true; }
+                if (bleft <= 0) { bleft = 0; exhausted = true; PTLOG(1); }
                 else { next_cnt = kBatch; next = atomicAdd(a.ticket, next_cnt); }
             }
             if (bleft == 0) {
                 if (npend > 0) continue;
+                // no tickets left: stay until the publisher has dealt with every streaming task of this CTA (it
+                // may still leave draw tasks), then stop the consumers
+                bool done = false;
+                for (uint32_t i = 0; i < kSpin && !done; ++i) {
+                    done = *(volatile int*)&S.pub_count == n_stream;      // read before the mailbox: its entries come first
+                    drain();
+                    if (!done) __nanosleep(100);
+                }
+                if (!done) atomicExch(a.wait_failed, 1);
                 const int stage = it % NST;
                 if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
                 S.desc[stage].phase = -1;
@@ -217,22 +292,22 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             }
             run = decode(bt, bleft);
             bt += run.cnt; bleft -= run.cnt;
-            if (!ready(run.ph, run_seq(run), false)) { S.pend[npend++] = run; continue; }
+            if (!ready(run.ph, run.wv, false)) { S.pend[npend++] = run; continue; }
         }
         // ---- the tasks of the run
-        const int ph = run.ph, wv = 0;
-        const int per_row = ph == 0 ? T : (ph == 2 ? T2 : 1), rows = ph == 0 ? NR : (ph == 2 ? K + 1 : 1);
+        const int ph = run.ph;
+        const int per_row = ph == 0 ? T : T2, rows = ph == 0 ? NR : K + 1;
         int s = run.off % per_row, r = (run.off / per_row) % rows;
         const int b = run.wv;                      // a run stays within one sequence
         int left = run.cnt;
         while (left > 0) {
             // the row's numbers
             TaskDesc d;
-            d.phase = ph; d.wave = wv; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f; d.c = 0.f;
+            d.phase = ph; d.wave = 0; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f; d.c = 0.f;
             d.P = no_row(); d.Q = no_row();
+            d.need = 0; d.bound = 0.f; d.tt = 0.0; d.base = 0.0;
             const char* row0 = nullptr; const char* row1 = nullptr;
             bool skip = false;
-            int* done = nullptr;
             if (ph == 0) {
                 const int L = len_of(R, b);
                 const bool is_target = r <= K;
@@ -240,7 +315,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
                 skip = is_target ? k > L : k >= L;
                 row0 = row_ptr(R, b, r);
-            } else if (ph == 2) {
+            } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
                 const int k = r;
                 const SeqInfo si = ld_cg(a.sinfo + b);
@@ -252,9 +327,10 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 if (k <= L) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
                 d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
-                done = &a.p2done[b];
                 const bool pair = k < L;
                 skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
+                // the sequence's second sweep: every half slice of the L row pairs, and of the bonus row if drawn from
+                d.need = T2 * (L + (si.draw_row == L ? 1 : 0));
                 if (!skip) {
                     d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
                     d.P = row_scale(sp);
@@ -264,26 +340,12 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 }
             }
             const int n_row = min(left, per_row - s);         // tasks of this run in this row
-            if (skip) {
-                if (done) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" :: "l"(done), "r"(n_row) : "memory");
-            } else {
+            if (!skip) {
                 const int sv = ph == 0 ? sv1 : sv2;
                 for (int i = 0; i < n_row; ++i) {
-                    const int stage = it % NST;
                     d.s = s + i; d.v0 = d.s * sv; d.nv = max(min(sv, R.nvec - d.v0), 0);
-                    if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
-                    S.desc[stage] = d;
-                    PLOG(1 + 10 * ph, it);
-                    const uint32_t bytes = (uint32_t)d.nv * 16u;
-                    if (row0 && bytes) {
-                        mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
-                        const unsigned long long pol = ph == 0 ? pol_keep : pol_drop;
-                        bulk_load(data + (size_t)stage * STAGE_BYTES, row0 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
-                        if (row1) bulk_load(data + (size_t)stage * STAGE_BYTES + STAGE_BYTES / 2, row1 + (int64_t)d.v0 * 16, bytes, &S.full[stage], pol);
-                    } else {
-                        mbar_arrive(&S.full[stage]);
-                    }
-                    ++it;
+                    issue(d, row0, row1, ph == 0 ? pol_keep : pol_drop);
+                    ++n_stream;
                 }
             }
             left -= n_row;
@@ -537,6 +599,193 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
     if (lane == 0) mbar_arrive(&S.pdone[stage]);
 }
 
+// ------------------------------------------------------------------ the draw
+// mass and sum of squares of half slice i of a sequence's draw rows (waits, bounded, for a part not there yet)
+__device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
+    unsigned long long w0 = 0, w1 = 0;
+    for (uint32_t k = 0; k < kSpin; ++k) {
+        w0 = __ldcg(a.dacc + 2 * i); w1 = __ldcg(a.dacc + 2 * i + 1);
+        if ((w0 & 15ull) != 0 && (w1 & 15ull) != 0) break;
+        __nanosleep(64);
+    }
+    if ((w0 & 15ull) == 0 || (w1 & 15ull) == 0) atomicExch(a.wait_failed, 1);
+    DPart d;
+    d.tot = (double)(w0 >> 4) * 3.469446951953614e-18;            // 2^-58
+    d.sq = (float)((double)(w1 >> 4) * 9.094947017729282e-13);    // 2^-40
+    d.pad = 1;
+    return d;
+}
+
+// Set-up of a sequence's draw, by the publisher warp that delivered the last partial of the sequence's second
+// sweep: TV of every draft position from the fixed-point sums, then the residual mass Z of the draw rows, the
+// target u * Z of the inverse CDF and the half slice that owns it.  The draw task goes into the CTA's mailbox:
+// the producer stages that half slice and the consumers find the token.
+__device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, int b) {
+    const RowArgs& R = a.r;
+    const int lane = threadIdx.x & 31;
+    const int K = R.K, NR = 2 * K + 1, L = len_of(R, b), T2 = 2 * a.T;
+    const SeqInfo si = ld_cg(a.sinfo + b);
+    if (si.n < 0) return;
+    const int k = si.draw_row;
+    const bool pair = k >= 0 && k < L;
+    // lane 0 will need the draw rows' records: asked for now, with everything else
+    RowStat sp, sq;
+    sp.inv_s = 0.0; sp.e = 0; sp.st = 0; sq = sp;
+    if (lane == 0 && k >= 0) { sp = ld_cg(a.rstat + (int64_t)b * NR + k); if (pair) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k); }
+    const float tau = tau_of(R, b);
+    if (lane < L && a.o.tv) {
+        // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
+        unsigned long long w = 0;
+        for (uint32_t i = 0; i < kSpin; ++i) {
+            w = __ldcg(a.tvacc + (int64_t)b * K + lane);
+            if ((int)(w & 0xffffull) >= T2) break;
+            __nanosleep(64);
+        }
+        if ((int)(w & 0xffffull) < T2) atomicExch(a.wait_failed, 1);
+        const float z = (float)((double)(w >> 16) * 9.094947017729282e-13);      // 2^-40
+        a.o.tv[(int64_t)b * K + lane] = fminf(fmaxf(z, 0.f), 1.f);
+    }
+    if (k < 0) return;
+    // the half slices' masses: lanes fetch them in parallel, lane 0 scans them in slice order
+    for (int s = lane; s < T2; s += 32) { const DPart dp = load_dpart(a, (int64_t)b * T2 + s); S.d1_tot[s] = dp.tot; S.d1_sq[s] = dp.sq; }
+    __syncwarp();
+    if (lane == 0) {
+        double Z = 0.0, sumsq = 0.0;
+        for (int s = 0; s < T2; ++s) { Z += S.d1_tot[s]; sumsq += (double)S.d1_sq[s]; }
+        const double Tt = (double)a.u_final[b] * Z;
+        double run = 0.0; int owner = -1; double base = 0.0;
+        for (int s = 0; s < T2; ++s) {
+            const double nx = run + S.d1_tot[s];
+            if (owner < 0 && Tt > run && Tt <= nx) { owner = s; base = run; }
+            run = nx;
+        }
+        if (!(Tt > 0.0)) owner = -1;
+        if (owner < 0) {
+            // no half slice owns the target (no residual mass, or u = 0): the fp64 re-draw decides
+            FbRec rec;
+            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0); rec.ep = sp.e; rec.eq = pair ? sq.e : 0;
+            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
+        } else {
+            // the mailbox has room for more draws than this CTA's unpublished tasks can bring; should it be full
+            // all the same, wait (bounded) for the producer
+            const int tail = S.mb_tail;
+            bool room = false;
+            for (uint32_t i = 0; i < kSpin && !room; ++i) {
+                room = tail - *(volatile int*)&S.mb_head < kMbox;
+                if (!room) __nanosleep(100);
+            }
+            if (!room) atomicExch(a.wait_failed, 1);
+            else {
+                DrawTask t;
+                t.tt = Tt; t.base = base; t.bound = (float)draw_bound(sumsq); t.c = temp_scale(tau).hi;
+                t.b = b; t.k = k; t.owner = owner; t.pair = pair ? 1 : 0;
+                t.P = row_scale(sp); t.Q = pair ? row_scale(sq) : no_row();
+                S.mbox[tail % kMbox] = t;
+                __threadfence_block();
+                *(volatile int*)&S.mb_tail = tail + 1;
+            }
+        }
+    }
+    __syncwarp();
+}
+
+// D: the token of a sequence from the half slice that owns the target of the inverse CDF (target row in the
+// first half of the stage, draft row in the second, like a P2 task).  The fp32 draw is kept when target and
+// running sum are further apart than the error bound on both sides of the token; else the sequence is listed
+// for the fp64 re-draw.
+template <int DT>
+__device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const TaskDesc& d, const unsigned char* data) {
+    constexpr int VEC = Elem<DT>::VEC;
+    const RowArgs& R = a.r;
+    WaveShared& S = PS.W;
+    float* vsum = PS.vsum;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = R.K, NR = 2 * K + 1, b = d.b, k = d.r;
+    const bool pair = (d.flags & 1) != 0;
+    const unsigned char* qdata = data + STAGE_BYTES / 2;
+    int found_y = -1, found_cert = 0;
+    if (!(d.flags & 4)) {
+        TempScale c; c.hi = d.c;
+        const RowScale SP = d.P, SQ = d.Q;
+        const int v0 = d.v0, nv = d.nv;
+        // per-vector residual mass, same arithmetic as phase P2
+        for (int v = tid; v < nv; v += PC) {
+            uint4 rp = lds16(data + (size_t)v * 16), rq = neg_inf_vec<DT>();
+            if (pair) rq = lds16(qdata + (size_t)v * 16);
+            const int gbase = (v0 + v) * VEC;
+            if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
+            float r[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
+            vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+        }
+        BEBOP_CTA_SYNC();
+        // contiguous ranges of vectors per thread, inclusive scan over threads
+        const int per = (nv + PC - 1) / PC;
+        const int vb = min(tid * per, nv), ve = min(vb + per, nv);
+        double mine = 0.0;
+        for (int v = vb; v < ve; ++v) mine += (double)vsum[v];
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { double t2 = shfl_up_d(incl, o); if (lane >= o) incl += t2; }
+        if (lane == 31) S.redd[warp] = incl;
+        BEBOP_CTA_SYNC();
+        double woff = 0.0;
+        for (int w = 0; w < warp; ++w) woff += S.redd[w];
+        double prev = shfl_up_d(incl, 1);
+        if (lane == 0) prev = 0.0;
+        const double Tt = d.tt, bound = (double)d.bound;
+        const double lower = d.base + woff + prev, upper = d.base + woff + incl;
+        if (lower < Tt && Tt <= upper) {
+            double C = lower;
+            for (int v = vb; v < ve && found_y < 0; ++v) {
+                const double nxt = C + (double)vsum[v];
+                if (Tt <= nxt) {
+                    uint4 rp = lds16(data + (size_t)v * 16), rq = neg_inf_vec<DT>();
+                    if (pair) rq = lds16(qdata + (size_t)v * 16);
+                    const int gbase = (v0 + v) * VEC;
+                    if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
+                    float r[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) r[i] = 0.f;
+                    residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
+                    double Cw = C;
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        if (found_y < 0) {
+                            const double r1 = (double)r[i];
+                            const double Cn = Cw + r1;
+                            if (r1 > 0.0 && Cn >= Tt) { found_y = gbase + i; found_cert = (Tt - Cw > bound) && (Cn - Tt >= bound); }
+                            Cw = Cn;
+                        }
+                    }
+                    break;
+                }
+                C = nxt;
+            }
+        }
+    }
+    // at most one thread should have found the token
+    const unsigned own = __ballot_sync(0xffffffffu, found_y >= 0);
+    if (lane == 0) S.redi[warp] = -1;
+    BEBOP_CTA_SYNC();
+    if (own && lane == (__ffs(own) - 1)) S.redi[warp] = (__popc(own) == 1 && found_cert) ? found_y : -2;
+    BEBOP_CTA_SYNC();
+    if (tid == 0) {
+        int y = -1, cnt = 0;
+        for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
+        if (cnt == 1 && y >= 0) a.o.out_tokens[(int64_t)b * (K + 1) + k] = y;
+        else {
+            FbRec rec;
+            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0);
+            rec.ep = ld_cg(a.rstat + (int64_t)b * NR + k).e;
+            rec.eq = pair ? ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k).e : 0;
+            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ publisher
 // One warp.  For every streaming task: wait for the eight warp partials, take them into registers,
 // hand the stage back, then merge (warp order, so the result does not depend on timing) and publish:
@@ -565,6 +814,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
         if (!mbar_wait(&S.pdone[stage], (pd_par >> stage) & 1u)) { if (lane == 0) atomicExch(a.wait_failed, 1); return; }
         pd_par ^= 1u << stage;
         const int b = S.desc[stage].b, r = S.desc[stage].r, sl = S.desc[stage].s, flags = S.desc[stage].flags;
+        const int need = S.desc[stage].need;
         const int w = lane & (WW - 1);
         const float f0 = S.wf[stage][0][w], f1 = S.wf[stage][1][w];
         const double dd = S.wd[stage][w];
@@ -598,6 +848,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
             }
         } else {
             float zz = 0.f, sq = 0.f; double tot = 0.0;
+            int run_d = 0;
 #pragma unroll
             for (int k = 0; k < WW; ++k) {
                 zz += __shfl_sync(0xffffffffu, f0, k); sq += __shfl_sync(0xffffffffu, f1, k); tot += __shfl_sync(0xffffffffu, dd, k);
@@ -611,9 +862,14 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
                     red_add_u64(wd, ((unsigned long long)__double2ll_rn(tot * kFixMass) << 4) | 1ull);
                     red_add_u64(wd + 1, ((unsigned long long)__double2ll_rn((double)sq * kFixTv) << 4) | 1ull);
                 }
-                asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" :: "l"(a.p2done + b) : "memory");
+                // the sequence's last partial starts the set-up of its draw
+                run_d = atomicAdd(a.p2done + b, 1) == need - 1;
             }
+            if (__shfl_sync(0xffffffffu, run_d, 0)) draw_setup_warp(a, S, b);
         }
+        // the producer stays until every streaming task has been dealt with here (mailbox entries come first)
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); *(volatile int*)&S.pub_count = *(volatile int*)&S.pub_count + 1; }
     }
 }
 
@@ -625,9 +881,13 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     unsigned char* data = smem;
     PipeShared& S = *reinterpret_cast<PipeShared*>(smem + (size_t)NST * STAGE_BYTES);
     const int tid = threadIdx.x;
+    // the re-draw kernel behind this one may be scheduled as CTAs of this one leave; it waits for this grid's
+    // completion before it reads anything (programmatic dependent launch)
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid == 0) PTLOG(0);
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], WW + 1); mbar_init(&S.pdone[i], WW); }
-        S.logn = 0;
+        S.logn = 0; S.mb_tail = 0; S.mb_head = 0; S.pub_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -645,17 +905,18 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (d.phase < 0) break;
         if (tid == 0) PLOG(2, it);
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
-        if (d.phase == 0) pipe_p1<DT>(a, S, d, sd, stage, it);
-        else if (d.phase == 2) pipe_p2<DT>(a, S, d, sd, stage, it);
+        if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage, it); if (tid == 0) PTLOG(6); }
+        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT>(a, S, d, sd, stage, it); if (tid == 0) PTLOG(5); }
         else {
-            // a D task's stage holds no logits: it is the task's scratch (per-vector masses, slice masses)
-            phase_d<DT>(a, S.W, d.b, reinterpret_cast<float*>(data + (size_t)stage * STAGE_BYTES));
+            if (tid == 0) PTLOG(2);
+            pipe_d<DT>(a, S, d, sd);
             BEBOP_CTA_SYNC();
-
+            if (tid == 0) PTLOG(3);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&S.empty[stage]);
     }
+    if (tid == 0) PTLOG(4);
 }
 
 // -----------------------------------------------------------------------------
@@ -719,7 +980,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;
     {
         const long long NR = 2 * a.K + 1;
-        const long long total = (long long)a.B * (NR * wp.T + (long long)(a.K + 1) * 2 * wp.T + 1);
+        const long long total = (long long)a.B * (NR * wp.T + (long long)(a.K + 1) * 2 * wp.T);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
         // Distance of the second sweep behind the first, in sequences.  The default is the whole batch (two full
@@ -734,7 +995,6 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
             if (lag > a.B) lag = a.B;
         }
         wa.lag = (int)lag;
-        wa.lag_d = (BEBOP_PIPE_LAGD > 0 && BEBOP_PIPE_LAGD < a.B) ? BEBOP_PIPE_LAGD : a.B;   // D tickets: behind P2, or all at the end
     }
     cudaError_t e = cudaMemsetAsync(w, 0, wp.zero_bytes, stream);
     if (e != cudaSuccess) return e;

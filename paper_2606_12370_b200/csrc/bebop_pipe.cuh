@@ -59,7 +59,7 @@ struct WaveArgs {
     unsigned long long* dacc;    // [B][2T][2] draw-row mass (2^-58) and sum of squares (2^-40), each << 4 | parts added
     unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
-    int ntickets, lag, lag_d;        // distance (sequences) of P2 behind P1 and of D behind P2
+    int ntickets, lag;               // distance (sequences) of P2 behind P1
     long long* trace;
     int T, slice_vecs, wave_seqs, nwaves;
 };
@@ -171,157 +171,6 @@ __device__ __forceinline__ void residual_vec(const uint4& rp, const uint4& rq, c
         const float q = FINE ? __fmaf_rn(aq, Q.inv_lo, __fmul_rn(aq, Q.inv)) : __fmul_rn(aq, Q.inv);
         r[i] = fmaxf(p - q, 0.f);
         if (sq) { *sq = fmaf(p, p, *sq); *sq = fmaf(q, q, *sq); }
-    }
-}
-
-// ------------------------------------------------------------------ phase D
-// mass and sum of squares of half slice i of a sequence's draw rows (waits, bounded, for a part not there yet)
-__device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
-    unsigned long long w0 = 0, w1 = 0;
-    for (uint32_t k = 0; k < kSpin; ++k) {
-        w0 = __ldcg(a.dacc + 2 * i); w1 = __ldcg(a.dacc + 2 * i + 1);
-        if ((w0 & 15ull) != 0 && (w1 & 15ull) != 0) break;
-        __nanosleep(64);
-    }
-    if ((w0 & 15ull) == 0 || (w1 & 15ull) == 0) atomicExch(a.wait_failed, 1);
-    DPart d;
-    d.tot = (double)(w0 >> 4) * 3.469446951953614e-18;            // 2^-58
-    d.sq = (float)((double)(w1 >> 4) * 9.094947017729282e-13);    // 2^-40
-    d.pad = 1;
-    return d;
-}
-constexpr int NTH_D = WT;            // threads that run phase D
-template <int DT>
-__device__ __forceinline__ void phase_d(const WaveArgs& a, WaveShared& S, int b, float* vsum) {
-    constexpr int VEC = Elem<DT>::VEC;
-    const RowArgs& R = a.r;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1, T = 2 * a.T, sv = a.slice_vecs >> 1;
-    const SeqInfo si = ld_cg(a.sinfo + b);
-    if (si.n < 0) return;
-    // TV of every draft position: slice parts in slice order
-    if (tid < L && a.o.tv) {
-        float z = 0.f;
-        // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
-        unsigned long long w = 0;
-        for (uint32_t i = 0; i < kSpin; ++i) {
-            w = __ldcg(a.tvacc + (int64_t)b * K + tid);
-            if ((int)(w & 0xffffull) >= T) break;
-            __nanosleep(64);
-        }
-        if ((int)(w & 0xffffull) < T) atomicExch(a.wait_failed, 1);
-        z = (float)((double)(w >> 16) * 9.094947017729282e-13);      // 2^-40
-        a.o.tv[(int64_t)b * K + tid] = fminf(fmaxf(z, 0.f), 1.f);
-    }
-    const int k = si.draw_row;
-    if (k < 0) return;
-    const bool pair = k < L;
-    // the half slices' masses: one thread each fetches its slice's words (in parallel), thread 0 then scans them
-    double* dtot = reinterpret_cast<double*>(vsum + SLICE_VECS / 2);     // behind the per-vector masses
-    float* dsq = reinterpret_cast<float*>(dtot + 2 * MAX_SLICES);
-    for (int s = tid; s < T; s += NTH_D) { const DPart dp = load_dpart(a, (int64_t)b * T + s); dtot[s] = dp.tot; dsq[s] = dp.sq; }
-    BEBOP_CTA_SYNC();
-    if (tid == 0) {
-        double Z = 0.0, sumsq = 0.0;
-        for (int s = 0; s < T; ++s) { Z += dtot[s]; sumsq += (double)dsq[s]; }
-        const double Tt = (double)a.u_final[b] * Z;
-        double run = 0.0; int owner = -1; double base = 0.0;
-        for (int s = 0; s < T; ++s) {
-            const double nx = run + dtot[s];
-            if (owner < 0 && Tt > run && Tt <= nx) { owner = s; base = run; }
-            run = nx;
-        }
-        S.owner_slice = (Tt > 0.0) ? owner : -1;
-        S.base = base; S.Ttarget = Tt; S.bound = draw_bound(sumsq);
-    }
-    BEBOP_CTA_SYNC();
-    const int s = S.owner_slice;
-    int found_y = -1, found_cert = 0;
-    if (s >= 0) {
-        const float tau = tau_of(R, b);
-        const TempScale c = temp_scale(tau);
-        const RowScale SP = row_scale(ld_cg(a.rstat + (int64_t)b * NR + k));
-        RowScale SQ = no_row();
-        if (pair) SQ = row_scale(ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k));
-        const int v0 = s * sv;
-        const int nv = max(min(sv, R.nvec - v0), 0);
-        const char* prow = row_ptr(R, b, k) + (int64_t)v0 * 16;
-        const char* qrow = pair ? row_ptr(R, b, K + 1 + k) + (int64_t)v0 * 16 : nullptr;
-        // per-vector residual mass, same arithmetic as phase P2
-        for (int v = tid; v < nv; v += WT) {
-            uint4 rp = ldg16(prow + (size_t)v * 16), rq = neg_inf_vec<DT>();
-            if (pair) rq = ldg16(qrow + (size_t)v * 16);
-            const int gbase = (v0 + v) * VEC;
-            if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
-            float r[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) r[i] = 0.f;
-            residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
-            vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-        }
-        BEBOP_CTA_SYNC();
-        // contiguous ranges of vectors per thread, inclusive scan over threads
-        const int per = (nv + WT - 1) / WT;
-        const int vb = min(tid * per, nv), ve = min(vb + per, nv);
-        double mine = 0.0;
-        for (int v = vb; v < ve; ++v) mine += (double)vsum[v];
-        double incl = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) { double t2 = shfl_up_d(incl, d); if (lane >= d) incl += t2; }
-        if (lane == 31) S.redd[warp] = incl;
-        BEBOP_CTA_SYNC();
-        double woff = 0.0;
-        for (int w = 0; w < warp; ++w) woff += S.redd[w];
-        double prev = shfl_up_d(incl, 1);
-        if (lane == 0) prev = 0.0;
-        const double Tt = S.Ttarget, bound = S.bound;
-        const double lower = S.base + woff + prev, upper = S.base + woff + incl;
-        if (lower < Tt && Tt <= upper) {
-            double C = lower;
-            for (int v = vb; v < ve && found_y < 0; ++v) {
-                const double nxt = C + (double)vsum[v];
-                if (Tt <= nxt) {
-                    uint4 rp = ldg16(prow + (size_t)v * 16), rq = neg_inf_vec<DT>();
-                    if (pair) rq = ldg16(qrow + (size_t)v * 16);
-                    const int gbase = (v0 + v) * VEC;
-                    if (gbase + VEC > R.V) { mask_tail<DT>(rp, R.V - gbase); mask_tail<DT>(rq, R.V - gbase); }
-                    float r[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) r[i] = 0.f;
-                    residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
-                    double Cw = C;
-#pragma unroll
-                    for (int i = 0; i < VEC; ++i) {
-                        if (found_y < 0) {
-                            const double r1 = (double)r[i];
-                            const double Cn = Cw + r1;
-                            if (r1 > 0.0 && Cn >= Tt) { found_y = gbase + i; found_cert = (Tt - Cw > bound) && (Cn - Tt >= bound); }
-                            Cw = Cn;
-                        }
-                    }
-                    break;
-                }
-                C = nxt;
-            }
-        }
-    }
-    // at most one thread should have found the token
-    const unsigned own = __ballot_sync(0xffffffffu, found_y >= 0);
-    if (lane == 0) S.redi[warp] = -1;
-    BEBOP_CTA_SYNC();
-    if (own && lane == (__ffs(own) - 1)) S.redi[warp] = (__popc(own) == 1 && found_cert) ? found_y : -2;
-    BEBOP_CTA_SYNC();
-    if (tid == 0) {
-        int y = -1, cnt = 0;
-        for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
-        if (cnt == 1 && y >= 0) a.o.out_tokens[(int64_t)b * (K + 1) + k] = y;
-        else {
-            FbRec rec;
-            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0);
-            rec.ep = ld_cg(a.rstat + (int64_t)b * NR + k).e;
-            rec.eq = pair ? ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k).e : 0;
-            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
-        }
     }
 }
 
