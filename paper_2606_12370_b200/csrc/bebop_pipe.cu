@@ -71,13 +71,17 @@ constexpr int STAGE_BYTES = PSLICE * 16;
 constexpr size_t kLagBytes = (size_t)BEBOP_PIPE_LAG_MB << 20;   // logits between the first sweep and the second
 constexpr int kPend = 4;                          // runs a producer may set aside
 #ifndef BEBOP_PIPE_BATCH
-#define BEBOP_PIPE_BATCH 2
+#define BEBOP_PIPE_BATCH 5
 #endif
-constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time in the first sweep
-#ifndef BEBOP_PIPE_BATCH2
-#define BEBOP_PIPE_BATCH2 2
+#ifndef BEBOP_PIPE_TAIL
+#define BEBOP_PIPE_TAIL 8
 #endif
-constexpr int kBatch2 = BEBOP_PIPE_BATCH2;        // ... and in the second sweep (more per-row numbers to fetch)
+constexpr int kTailZone = BEBOP_PIPE_TAIL;        // the last kTailZone tickets per CTA are claimed kBatchTail at a time
+#ifndef BEBOP_PIPE_BATCH_TAIL
+#define BEBOP_PIPE_BATCH_TAIL 2
+#endif
+constexpr int kBatchTail = BEBOP_PIPE_BATCH_TAIL;
+constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time (measured: 4 to 6 alike, 2 and 8 slower)
 constexpr double kFixTv = 1099511627776.0;             // 2^40: fixed point of TV parts and sums of squares
 constexpr double kFixMass = 288230376151711744.0;      // 2^58: fixed point of the draw-row mass
 constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
@@ -253,11 +257,11 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             issue(d, row_ptr(R, t.b, t.k), t.pair ? row_ptr(R, t.b, K + 1 + t.k) : nullptr, pol_drop);
         }
     };
+    const int tail_zone = (int)gridDim.x * kTailZone;
     int npend = 0;
     bool exhausted = false;
     int bt = 0, bleft = 0;                         // tickets of the claimed batch not yet turned into runs
-    int next_cnt = kBatch;                         // tickets of the claim in flight
-    int next = atomicAdd(a.ticket, next_cnt);
+    int last_seen = 0;                             // the latest ticket this CTA has seen handed out
     for (;;) {
         drain();
         // ---- next run
@@ -269,9 +273,11 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             for (int i = 0; i < npend; ++i) S.pend[i] = S.pend[i + 1];
         } else {
             if (bleft == 0 && !exhausted) {
-                bt = next; bleft = min(next_cnt, a.ntickets - bt);
+                // (claiming a batch ahead of need gained nothing and made the CTAs finish further apart)
+                const int cnt = (a.ntickets - last_seen <= tail_zone) ? kBatchTail : kBatch;
+                bt = atomicAdd(a.ticket, cnt); bleft = min(cnt, a.ntickets - bt);
+                last_seen = bt;
                 if (bleft <= 0) { bleft = 0; exhausted = true; PTLOG(1); }
-                else { next_cnt = kBatch; next = atomicAdd(a.ticket, next_cnt); }
             }
             if (bleft == 0) {
                 if (npend > 0) continue;
