@@ -35,7 +35,7 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-KERNEL_OF_PATH = {0: "k_pipe", 2: "k_pipe", 3: "k_row"}
+KERNEL_OF_PATH = {0: "k_pipe"}
 
 
 def ncu_traffic(kernel):

@@ -9,7 +9,7 @@ namespace {
 
 // Test hook: route bebop_verify through the general (split-row) path even where the fused
 // kernel applies, so that both paths are covered by the parity tests.
-int g_path = 0;   // 0: the default order of kernels; 1: general kernels only; 2: pipelined kernel; 3: row kernel
+int g_path = 0;   // 0: pipelined kernel where it applies, else the general kernels; 1: general kernels only
 
 // Built-in scratch of bebop_tv_static: one array per device the module is loaded on.  Nothing in it
 // has to start at zero (every partial is written before it is read).
@@ -100,9 +100,7 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 3 && row_supported(a))
-        e = row_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    if (e == cudaSuccess && !launched && (g_path == 0 || g_path == 2) && pipe_supported(a))
+    if (g_path == 0 && pipe_supported(a))
         e = pipe_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
     if (e == cudaSuccess && !launched) e = general_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;

@@ -60,11 +60,4 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched);
 
-// Row kernel (bebop_row.cu): groups of CTAs keep a row pair in shared memory between the softmax pass and the
-// residual pass, so that every logit is read from HBM once; same contract.
-bool row_supported(const RowArgs& a);
-cudaError_t row_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
-                       const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                       cudaStream_t stream, bool* launched);
-
 }  // namespace bebop

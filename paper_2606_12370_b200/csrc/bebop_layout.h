@@ -27,39 +27,7 @@ struct WavePlan {
     size_t off_part, off_rstat, off_dpart, off_tvacc, off_sinfo, total;
 };
 
-// Workspace of the row kernel (bebop_row.cu): a group of G CTAs holds one row pair in shared memory, rank r
-// the vectors [r * SV, r * SV + SV) of both rows, in NCH chunks of kRowChunkVecs vectors.
-constexpr int kRowChunkVecs = 512;       // 16-byte vectors per chunk and row (two per consumer thread)
-constexpr int kRowMaxChunks = 5;
-constexpr int kRowMaxGroup = 32;
-struct RowPlan {
-    int G, SV, NCH;                      // 0: the shape is not supported
-    size_t off_grec;                     // 16-byte records [tasks][G][2]: the CTAs' softmax partials of a row pair
-    size_t off_arec;                     // 16-byte records [B][K]: p(x), q(x) and the accept decision of a position
-    size_t off_cacc;                     // u64 [B][K+1][G*NCH][2]: chunk masses and sums of squares, fixed point
-    size_t off_seqcnt;                   // int [B]: CTA-level row tasks finished
-    size_t total;
-};
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-static inline RowPlan make_row_plan(int B, int K, int nvec) {
-    RowPlan r;
-    r.G = 0; r.SV = 0; r.NCH = 0; r.off_grec = r.off_arec = r.off_cacc = r.off_seqcnt = 0; r.total = 0;
-    // groups as small as four chunks per CTA allow (then three CTAs of a row-pair slice each fit one SM)
-    int G = (nvec + 4 * kRowChunkVecs - 1) / (4 * kRowChunkVecs);
-    if (G < 1) G = 1;
-    if (G > kRowMaxGroup) return r;
-    r.G = G;
-    r.SV = ((((nvec + G - 1) / G) + 15) / 16) * 16;
-    r.NCH = (r.SV + kRowChunkVecs - 1) / kRowChunkVecs;
-    size_t o = 0;
-    r.off_grec = o;   o += align256(32 * (size_t)B * (K + 1) * G);
-    r.off_arec = o;   o += align256(16 * (size_t)B * (K > 0 ? K : 1));
-    r.off_cacc = o;   o += align256(16 * (size_t)B * (K + 1) * G * r.NCH);
-    r.off_seqcnt = o; o += align256(sizeof(int) * (size_t)B);
-    r.total = o;
-    return r;
-}
-
 struct Plan {
     int B, K, V, dt;
     int nvec;        // 16-byte vectors per row (last one possibly ragged)
@@ -75,7 +43,6 @@ struct Plan {
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
     size_t off_fb;      // 16-byte records [B]: the sequences whose draw goes to fp64
     size_t off_wave;    // workspace of the pipelined kernel
-    size_t off_row;     // workspace of the row kernel
     size_t total;
 };
 
@@ -141,7 +108,6 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_fb = o;     o = align256(o + 16 * (size_t)B);
     {
         p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
-        p.off_row = o;    o = align256(o + make_row_plan(B, K, p.nvec).total);
     }
     p.total = o;
     return p;
