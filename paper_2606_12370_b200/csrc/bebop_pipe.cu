@@ -1,11 +1,12 @@
 // Pipelined kernel: the hot path of bebop_verify as one persistent, ticket-scheduled kernel with the
 // data movement and the bookkeeping taken off the compute warps.
 //
-// The work is a queue of tickets in three blocks: P1 (softmax partial of one slice of one row) for
-// every row, then P2 (TV and residual mass of one half slice of a row pair) for every position, then D
-// (the fast draw with its certificate) for every sequence; sequences ascending.  Phase A -- merging a
-// row's partials, and the accept scan of a sequence -- has no tickets: it runs in the publisher warp
-// that completes the row / the sequence, long before the second sweep asks for its results.
+// The work is a queue of tickets in two blocks: P1 (softmax partial of one slice of one row) for
+// every row, then P2 (TV and residual mass of one half slice of a row pair) for every position;
+// sequences ascending.  Phase A -- merging a row's partials, and the accept scan of a sequence -- has no
+// tickets: it runs in the publisher warp that completes the row / the sequence, long before the second
+// sweep asks for its results.  Nor has the draw: the publisher warp that completes a sequence's second
+// sweep sets the draw up and hands it to its own CTA as a task D (the fast draw with its certificate).
 //
 // A CTA is eight consumer warps, a producer warp and a publisher warp around a ring of shared-memory
 // stages.  The producer's first lane claims tickets, decodes them into runs of consecutive slices,
@@ -165,9 +166,6 @@ __device__ __forceinline__ unsigned long long l2_policy(bool keep) {
     return p;
 }
 __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
-__device__ __forceinline__ void release_add(int* p) {
-    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" :: "l"(p) : "memory");
-}
 
 
 #ifdef BEBOP_TRACE

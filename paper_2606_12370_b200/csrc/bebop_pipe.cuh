@@ -1,13 +1,8 @@
-// Device code of the verify path that does not depend on how a CTA gets its data: workspace records,
-// small helpers, the residual arithmetic, the draw bound and phase D (the fast draw with its certificate).
-// The including file defines BEBOP_CTA_SYNC() (the barrier of the threads that run phase D) first.
+// Device code shared by the pipelined kernel and the re-draw kernels: workspace records, small helpers,
+// the residual arithmetic and the draw bound.
 #pragma once
 #include "bebop_kernels.h"
 #include "bebop_ptx.cuh"
-
-#ifndef BEBOP_CTA_SYNC
-#error "define BEBOP_CTA_SYNC() before including bebop_pipe.cuh"
-#endif
 
 namespace bebop {
 

@@ -1,28 +1,8 @@
-// The fp64 re-draw of the sequences whose fast draw did not clear its error bound, the kernel that turns
-// an expired device-side wait into a status bit, and the hooks that time and trace the main kernel.
-#define BEBOP_CTA_SYNC() __syncthreads()
+// The fp64 re-draw of the sequences whose fast draw did not clear its error bound (its first kernel also turns
+// an expired device-side wait into a status bit), and the hooks that time and trace the main kernel.
 #include "bebop_pipe.cuh"
 
 namespace bebop {
-
-#ifdef BEBOP_TRACE
-// timeline of the re-draw kernels: [2i] earliest, [2i+1] latest global-timer stamp of event i over all threads that log it
-__device__ unsigned long long g_rd_trace[32];
-__device__ __forceinline__ void rd_log(int i) {
-    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    atomicMin(&g_rd_trace[2 * i], t); atomicMax(&g_rd_trace[2 * i + 1], t);
-}
-#define RDLOG(i) do { if (threadIdx.x == 0) rd_log(i); } while (0)
-extern "C" void bebop_debug_redraw_trace(unsigned long long* host32, int reset) {
-    if (reset) {
-        unsigned long long init[32];
-        for (int i = 0; i < 16; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
-        cudaMemcpyToSymbol(g_rd_trace, init, sizeof(init));
-    } else cudaMemcpyFromSymbol(host32, g_rd_trace, 32 * sizeof(unsigned long long));
-}
-#else
-#define RDLOG(i) do { } while (0)
-#endif
 
 namespace {
 
@@ -130,11 +110,9 @@ __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
     __shared__ double tab[XTAB];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // launched as a programmatic dependent of the main kernel: set up, then wait for that grid's completion
-    RDLOG(0);
     x_exp2_table(tab);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    RDLOG(1);
     const int XT = 4 * a.T, items = *a.fb_count * XT;
     // a wait of the main kernel that gave up: every row's status says so
     if (a.o.row_status && *a.wait_failed) {
@@ -147,10 +125,7 @@ __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
         XRow d;
         x_row(a, slot, &d);
         float fp[XNU][VEC], fq[XNU][VEC];
-        RDLOG(2);
         x_load<DT>(a, d, s, fp, fq);
-        if (fp[0][0] == 12345.f) RDLOG(15);
-        RDLOG(3);
         double sa = 0.0, sb = 0.0;
 #pragma unroll
         for (int u = 0; u < XNU; ++u) {
@@ -161,8 +136,6 @@ __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
             }
         }
         sa = warp_sum(sa); sb = warp_sum(sb);
-        if (sa == 12345.0) RDLOG(15);
-        RDLOG(4);
         __syncthreads();
         if (lane == 0) { sh[0][warp] = sa; sh[1][warp] = sb; }
         __syncthreads();
@@ -171,7 +144,6 @@ __global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
             for (int w = 0; w < WW; ++w) { ta += sh[0][w]; tb += sh[1][w]; }
             a.xsum[(int64_t)d.b * XT + s] = make_double2(ta, tb);
         }
-        RDLOG(5);
     }
 }
 
@@ -208,10 +180,8 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
     __shared__ double tab[XTAB];
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    RDLOG(6);
     x_exp2_table(tab);
     asm volatile("griddepcontrol.wait;" ::: "memory");      // programmatic dependent of k_redraw_sum
-    RDLOG(7);
     const int K = R.K, XT = 4 * a.T, items = *a.fb_count * XT;
     const int qv = a.slice_vecs >> 2, cw = (qv + WW - 1) / WW;
     if ((int)blockIdx.x >= items) return;
@@ -227,8 +197,6 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
         for (int t = lane; t < XT; t += 32) { const double2 x = a.xsum[(int64_t)b * XT + t]; Sa += x.x; Sb += x.y; }
         Sa = warp_sum(Sa); Sb = warp_sum(Sb);
         d.ip = 1.0 / Sa; d.iq = d.pair ? 1.0 / Sb : 0.0;
-        if (d.ip == 12345.0) RDLOG(15);
-        RDLOG(8);
         if (d.pair) {     // a bonus row needs no mass pass: its masses are sums of exponentials over Sa
             float fp[XNU][VEC], fq[XNU][VEC];
             x_load<DT>(a, d, s, fp, fq);
@@ -242,14 +210,12 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
             if (lane == 0) a.xmass[((int64_t)b * XT + s) * WW + warp] = m;
         }
         __syncthreads();
-        RDLOG(9);
         if (tid == 0) {
             __threadfence();
             S.last = atomicAdd(a.xdone + slot, 1) == XT - 1;
         }
         __syncthreads();
         if (!S.last) continue;
-        RDLOG(10);
         __threadfence();
 
         // ---- pick.  Stage 1: quarter slice from the slice masses.
@@ -282,7 +248,6 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
         }
         __syncthreads();
         const int qs = S.sel;
-        RDLOG(11);
         // Stage 2: warp chunk inside the quarter slice (residual: stored; plain softmax row: evaluated now)
         const int p0 = qs * qv, pn = max(min(qv, R.nvec - p0), 0);
         double wm = 0.0;
@@ -309,7 +274,6 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
             S.tok_first = 0x7fffffff; S.tok_last = -1;
         }
         __syncthreads();
-        RDLOG(12);
         // Stage 3: the tokens of the chunk, `per` consecutive tokens per thread, scanned in token order
         const int e0 = (p0 + S.chunk * cw) * VEC;                                 // first token of the chunk
         const int e1 = min(min((p0 + min((S.chunk + 1) * cw, pn)) * VEC, R.V), e0 + 4 * WT);
@@ -350,7 +314,6 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
         if (lastpos >= 0) atomicMax(&S.tok_last, lastpos);
         __syncthreads();
         if (tid == 0) a.o.out_tokens[(int64_t)b * (K + 1) + d.k] = S.tok_first != 0x7fffffff ? S.tok_first : S.tok_last;
-        RDLOG(13);
         __syncthreads();
     }
 }
