@@ -202,6 +202,12 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     // the run of consecutive tasks of one sequence and phase that starts at ticket t, at most `want` tasks;
     // Run.wv is the sequence, Run.off the offset inside the sequence's block of that phase
     auto decode = [&](int t, int want) {
+        if (W >= B && f_next <= t) {
+            // two full sweeps: the block follows from one division (a CTA's next tickets are some thirty blocks
+            // on: stepping there one block at a time was most of what the producer did between two runs)
+            blk = t < B * c0 ? t / c0 : B + (t - B * c0) / c2;
+            f_here = before(blk); f_next = before(blk + 1);
+        }
         while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
         Run r;
         int o = t - f_here, room;
