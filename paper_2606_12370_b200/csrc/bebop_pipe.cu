@@ -165,6 +165,14 @@ __device__ __forceinline__ unsigned long long l2_policy(bool keep) {
     else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
+// n / d for 0 <= n < 2^31, 0 < d, with inv = 1.0 / d: a multiplication and a correction instead of the
+// forty-odd instructions of an integer division (the producer is one thread: its instructions are its time)
+__device__ __forceinline__ int div_by(int n, int d, double inv) {
+    int q = __double2int_rz((double)n * inv);
+    const int r = n - q * d;
+    if (r >= d) ++q; else if (r < 0) --q;
+    return q;
+}
 __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
 
 
@@ -188,6 +196,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
     const int B = R.B;
     const int c0 = NR * T, c2 = (K + 1) * T2;
+    const double inv_c0 = 1.0 / c0, inv_c2 = 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
     // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
     // exists).  With W = B (the default) that is all of P1, then all of P2: two full sweeps, sequences ascending,
@@ -205,7 +214,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         if (W >= B && f_next <= t) {
             // two full sweeps: the block follows from one division (a CTA's next tickets are some thirty blocks
             // on: stepping there one block at a time was most of what the producer did between two runs)
-            blk = t < B * c0 ? t / c0 : B + (t - B * c0) / c2;
+            blk = t < B * c0 ? div_by(t, c0, inv_c0) : B + div_by(t - B * c0, c2, inv_c2);
             f_here = before(blk); f_next = before(blk + 1);
         }
         while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
@@ -306,8 +315,10 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         }
         // ---- the tasks of the run
         const int ph = run.ph;
-        const int per_row = ph == 0 ? T : T2, rows = ph == 0 ? NR : K + 1;
-        int s = run.off % per_row, r = (run.off / per_row) % rows;
+        const int per_row = ph == 0 ? T : T2;
+        // a run starts inside its sequence's block of the phase: row and slice from the offset (rows * per_row tasks)
+        int r = div_by(run.off, per_row, ph == 0 ? inv_T : inv_T2);
+        int s = run.off - r * per_row;
         const int b = run.wv;                      // a run stays within one sequence
         int left = run.cnt;
         while (left > 0) {
