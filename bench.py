@@ -247,6 +247,27 @@ def run_ours(args):
     clocks = sampler.summary(t0, t1)
     launches_per_call = 6 if args.path == 1 else 3      # main kernel, 2 fp64 re-draw kernels | 6 general kernels
 
+    # the same call without a TV output (the second sweep then reads only the rows a token is drawn from): not the
+    # headline, which emits TV; reported beside it
+    notv_steps = max(1, min(steps, 200))
+    out_notv = {k: v for k, v in out.items() if k != "tv"}
+
+    def step_notv():
+        return P.bebop_verify(x["target"], x["draft"], x["draft_tokens"], x["u_accept"], x["u_final"],
+                              draft_len=x["draft_len"], temperature=x["temperature"],
+                              temperature_all=x["temperature_all"], out=out_notv, workspace=ws, want_tv=False)
+
+    for _ in range(3):
+        step_notv()
+    barrier()
+    n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0.record()
+    for _ in range(notv_steps):
+        step_notv()
+    n1.record()
+    barrier()
+    notv_ms = n0.elapsed_time(n1) / notv_steps
+
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))
     host = {k: x[k].cpu().pin_memory() for k in ("target", "draft", "draft_tokens", "u_accept", "u_final")}
@@ -276,7 +297,7 @@ def run_ours(args):
 
     # max over ranks
     from paper_2606_12370_b200.shard import max_over_ranks
-    ms, e2e_s = max_over_ranks([ms, e2e_s], dist, dev)
+    ms, e2e_s, notv_ms = max_over_ranks([ms, e2e_s, notv_ms], dist, dev)
     sampler.stop()
 
     if rank == 0:
@@ -298,6 +319,8 @@ def run_ours(args):
             "e2e": {"value": world * positions / e2e_s, "unit": "positions/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3},
             "gpu_launches": steps * launches_per_call,
+            "without_tv": {"value": world * positions / (notv_ms * 1e-3), "unit": "positions/s", "ms_per_step": notv_ms,
+                           "steps": notv_steps, "note": "same call with tv = NULL; not the headline"},
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,
             "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, B == 256, KERNEL_OF_PATH.get(args.path, "general kernels"), len(pairs)),
         }

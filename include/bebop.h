@@ -86,7 +86,8 @@ size_t bebop_workspace_bytes(int B, int K, int V, bebop_dtype_t dt);
  * temperature   [B] fp32, or NULL -> temperature_all (> 0) for every row
  * u_accept [B,K], u_final [B] : fp32 uniforms in the open interval (0,1)
  * accept_len [B], out_tokens [B,K+1] (x_1..x_n, y, then -1) : int32 outputs
- * tv, p_draft, q_draft [B,K] fp32 outputs, each may be NULL (0 beyond draft_len)
+ * tv, p_draft, q_draft [B,K] fp32 outputs, each may be NULL (0 beyond draft_len).  With tv = NULL the
+ *   residuals are formed only at the position a token is drawn from, and the call reads that much less.
  * row_status [B] int32 output, may be NULL
  */
 bebop_status_t bebop_verify(

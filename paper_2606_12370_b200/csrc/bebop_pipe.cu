@@ -195,7 +195,8 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     const RowArgs& R = a.r;
     const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
     const int B = R.B;
-    const int c0 = NR * T, c2 = (K + 1) * T2;
+    // (a caller that asks for no TV needs the second sweep over one row per sequence only: the one a token is drawn from)
+    const int c0 = NR * T, c2 = (a.o.tv ? K + 1 : 1) * T2;
     const double inv_c0 = 1.0 / c0, inv_c2 = 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
     // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
@@ -338,8 +339,9 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 row0 = row_ptr(R, b, r);
             } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
-                const int k = r;
                 const SeqInfo si = ld_cg(a.sinfo + b);
+                const int k = a.o.tv ? r : max(si.draw_row, 0);
+                d.r = k;
                 RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 RowStat sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + min(k, K - 1));
                 const int L = len_of(R, b);
@@ -352,6 +354,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
                 // the sequence's second sweep: every half slice of the L row pairs, and of the bonus row if drawn from
                 d.need = T2 * (L + (si.draw_row == L ? 1 : 0));
+                if (!a.o.tv) d.need = T2;
                 if (!skip) {
                     d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
                     d.P = row_scale(sp);
@@ -1001,7 +1004,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;
     {
         const long long NR = 2 * a.K + 1;
-        const long long total = (long long)a.B * (NR * wp.T + (long long)(a.K + 1) * 2 * wp.T);
+        const long long total = (long long)a.B * (NR * wp.T + (long long)(o.tv ? a.K + 1 : 1) * 2 * wp.T);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
         // Distance of the second sweep behind the first, in sequences.  The default is the whole batch (two full

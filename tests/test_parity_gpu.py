@@ -184,6 +184,19 @@ def test_optional_outputs_may_be_null():
     assert torch.equal(a["accept_len"], b["accept_len"]) and torch.equal(a["out_tokens"], b["out_tokens"])
 
 
+def test_without_tv_same_tokens_on_a_large_vocabulary():
+    """Without a TV output the second sweep reads only the rows a token is drawn from: tokens, accept
+    lengths, probabilities and status must not change (ragged lengths, bonus and residual draws)."""
+    cfg = G.Config("notv", 24, 4, 40000, "bf16", 3.0, True, 1.0, 1.0, seed=21)
+    x = G.make_inputs(cfg, DEV)
+    x["draft_len"] = torch.tensor([(i * 7) % 5 for i in range(cfg.B)], dtype=torch.int32, device=DEV)
+    a = run_verify(x)
+    b = run_verify(x, want_tv=False)
+    assert b["tv"] is None
+    for k in ("accept_len", "out_tokens", "p_draft", "q_draft", "row_status"):
+        assert torch.equal(a[k], b[k]), k
+
+
 def test_deterministic_and_stream_ordered():
     cfg = G.Config("det", 16, 3, 32768, "bf16", 3.0, True, 1.0, 1.0, seed=8)
     x = G.make_inputs(cfg, DEV)
