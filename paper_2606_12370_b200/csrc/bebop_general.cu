@@ -10,7 +10,6 @@ namespace bebop {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kListSlots = 32;   // sequences in flight per pass of the list-driven draw
 constexpr float kNegInf = -INFINITY;
 
 __device__ __forceinline__ float tau_of(const RowArgs& a, int b) {
@@ -726,22 +725,6 @@ cudaError_t general_verify(const RowArgs& a, const Plan& p, const int32_t* draft
     LAUNCH_DT(a.dt, k_draw_stats, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats, all);
     LAUNCH_DT(a.dt, k_draw_mass, (unsigned)((int64_t)a.B * p.nsplit_d), kThreads, stream, a, stop, p.nsplit_d, dstats, dmass, all);
     LAUNCH_DT(a.dt, k_draw_pick, (unsigned)a.B, kThreads, stream, a, stop, p.nsplit_d, dstats, dmass, u_final, o, all);
-    return cudaGetLastError();
-}
-
-// fp64 draw for the sequences a device-side list names (the fused kernel's uncertain draws).
-// stop[b] holds the stop position of every listed sequence.  The split count is fixed at
-// kListSplit so that a handful of sequences still spreads over the whole GPU.
-cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
-                              const int* list, const int* count, cudaStream_t stream) {
-    int* stop = reinterpret_cast<int*>(ws + p.off_stop);
-    double2* dstats = reinterpret_cast<double2*>(ws + p.off_dstats);
-    double* dmass = reinterpret_cast<double*>(ws + p.off_dmass);
-    DrawList dl{list, count};
-    const int slots = a.B < kListSlots ? a.B : kListSlots;
-    LAUNCH_DT(a.dt, k_draw_stats, (unsigned)(slots * p.nsplit_l), kThreads, stream, a, stop, p.nsplit_l, dstats, dl);
-    LAUNCH_DT(a.dt, k_draw_mass, (unsigned)(slots * p.nsplit_l), kThreads, stream, a, stop, p.nsplit_l, dstats, dmass, dl);
-    LAUNCH_DT(a.dt, k_draw_pick, (unsigned)slots, kThreads, stream, a, stop, p.nsplit_l, dstats, dmass, u_final, o, dl);
     return cudaGetLastError();
 }
 

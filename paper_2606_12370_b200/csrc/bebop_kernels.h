@@ -41,9 +41,6 @@ cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft
                            int32_t* accept_len, int32_t* out_tokens, int32_t* row_status, char* ws,
                            cudaStream_t stream);
 
-cudaError_t general_draw_list(const RowArgs& a, const Plan& p, const float* u_final, VerifyOut o, char* ws,
-                              const int* list, const int* count, cudaStream_t stream);
-
 void wave_set_trace(long long* p);                            // trace buffer of the main kernel (BEBOP_TRACE builds)
 void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the main kernel of the next calls (nullptr: off)
 

@@ -19,10 +19,8 @@ struct alignas(16) FbRec {
 };
 constexpr size_t kFbCountOffset = 128;   // int: sequences listed for the fp64 re-draw, inside the zeroed head of the workspace
 struct WavePlan {
-    int T, slice_vecs;     // slices per row, vectors per slice (multiple of 8)
-    int wave_seqs, nwaves; // sequences per wave, waves
-    int lag;               // waves of stats work scheduled between a phase and the phase it depends on
-    size_t off_p1done, off_adone, off_p2done, off_xdone, off_rowcnt, zero_bytes;
+    int T, slice_vecs;     // slices per row, vectors per slice (multiple of 16)
+    size_t off_p1done, off_p2done, off_xdone, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
     size_t off_part, off_rstat, off_dpart, off_tvacc, off_sinfo, total;
 };
@@ -53,16 +51,8 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.T = (nvec + slice_cap - 1) / slice_cap; if (w.T < 1) w.T = 1;
     w.slice_vecs = (((nvec + w.T - 1) / w.T) + 15) & ~15;   // halves (phase P2) stay 128-byte aligned
     const size_t NR = (size_t)(2 * K + 1);
-    const size_t seq_bytes = NR * (size_t)nvec * 16;
-    size_t ws = ((size_t)18 << 20) / (seq_bytes ? seq_bytes : 1);
-    if (ws < 1) ws = 1;
-    if (ws > (size_t)B) ws = (size_t)B;
-    w.wave_seqs = (int)ws;
-    w.nwaves = (B + w.wave_seqs - 1) / w.wave_seqs;
-    w.lag = 2;
     size_t o = 256;                                           // ticket, wait flag; at kFbCountOffset the re-draw count
     w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per sequence: rows merged
-    w.off_adone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_rowcnt = o; o += align256(sizeof(int) * (size_t)B * NR);

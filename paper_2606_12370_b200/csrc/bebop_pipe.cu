@@ -88,8 +88,8 @@ constexpr double kFixMass = 288230376151711744.0;      // 2^58: fixed point of t
 constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
 
 struct __align__(16) TaskDesc {
-    int phase;        // 0 P1, 1 A, 2 P2, 3 D, -1: no more tasks
-    int wave, b, r;   // r: row (P1) or draft position (P2)
+    int phase;        // 0 P1, 2 P2, 3 D, -1: no more tasks
+    int b, r;         // sequence; row (P1) or draft position (P2, D)
     int s, v0, nv;    // slice, its first vector, its vectors
     int flags;        // bit 0: row pair (else bonus row alone), bit 1: the pair a token is drawn from,
                       // bit 2 (D): no half slice owns the target, the draw goes to the fp64 re-draw
@@ -264,7 +264,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             ++mb_head;
             *(volatile int*)&S.mb_head = mb_head;
             TaskDesc d;
-            d.phase = 3; d.wave = 0; d.b = t.b; d.r = t.k; d.s = t.owner; d.flags = (t.pair ? 1 : 0) | 2;
+            d.phase = 3; d.b = t.b; d.r = t.k; d.s = t.owner; d.flags = (t.pair ? 1 : 0) | 2;
             d.v0 = t.owner * sv2; d.nv = max(min(sv2, R.nvec - d.v0), 0);
             d.tau = 1.f; d.c = t.c; d.P = t.P; d.Q = t.Q; d.need = 0;
             d.bound = t.bound; d.tt = t.tt; d.base = t.base;
@@ -325,7 +325,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         while (left > 0) {
             // the row's numbers
             TaskDesc d;
-            d.phase = ph; d.wave = 0; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f; d.c = 0.f;
+            d.phase = ph; d.b = b; d.r = r; d.s = 0; d.v0 = 0; d.nv = 0; d.flags = 0; d.tau = 1.f; d.c = 0.f;
             d.P = no_row(); d.Q = no_row();
             d.need = 0; d.bound = 0.f; d.tt = 0.0; d.base = 0.0;
             const char* row0 = nullptr; const char* row1 = nullptr;
@@ -493,7 +493,7 @@ __device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long
 // P1: softmax partial (E, S) of one slice of one row, from shared memory.
 template <int DT>
 __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
-                                        int stage, int it) {
+                                        int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -560,7 +560,7 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
 // row in the second.
 template <int DT>
 __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
-                                        int stage, int it) {
+                                        int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / (2 * PC);
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -929,8 +929,8 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (d.phase < 0) break;
         if (tid == 0) PLOG(2, it);
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
-        if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage, it); if (tid == 0) PTLOG(6); }
-        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT>(a, S, d, sd, stage, it); if (tid == 0) PTLOG(5); }
+        if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
+        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
         else {
             if (tid == 0) PTLOG(2);
             pipe_d<DT>(a, S, d, sd);
@@ -1001,7 +1001,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.tvacc = reinterpret_cast<unsigned long long*>(w + wp.off_tvacc);
     wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
     wa.trace = g_wave_trace;
-    wa.T = wp.T; wa.slice_vecs = wp.slice_vecs; wa.wave_seqs = wp.wave_seqs; wa.nwaves = wp.nwaves;
+    wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
     {
         const long long NR = 2 * a.K + 1;
         const long long total = (long long)a.B * (NR * wp.T + (long long)(o.tv ? a.K + 1 : 1) * 2 * wp.T);

@@ -46,8 +46,8 @@ struct WaveArgs {
     // workspace
     int* ticket;          // [1]
     int* wait_failed;     // [1]
-    int* p1done;          // [nwaves]
-    int* p2done;          // [nwaves]
+    int* p1done;          // [B] rows of the sequence merged
+    int* p2done;          // [B] partials of the sequence's second sweep delivered
     int* rowcnt;          // [B][2K+1] pipelined kernel: softmax partials delivered per row
     P1Part* part;         // [B][2K+1][T]
     RowStat* rstat;       // [B][2K+1]
@@ -56,7 +56,7 @@ struct WaveArgs {
     SeqInfo* sinfo;       // [B]
     int ntickets, lag;               // distance (sequences) of P2 behind P1
     long long* trace;
-    int T, slice_vecs, wave_seqs, nwaves;
+    int T, slice_vecs;
 };
 
 __device__ __forceinline__ float tau_of(const RowArgs& a, int b) { return a.temperature ? a.temperature[b] : a.temperature_all; }
