@@ -109,7 +109,8 @@ struct DrawTask {
     int b, k, owner, pair;
     RowScale P, Q;
 };
-constexpr int kMbox = 8;                     // mailbox entries: more than the tasks a CTA can have unpublished
+constexpr int kMbox = 16;                    // mailbox entries: more than the tasks a CTA can have unpublished
+static_assert(kMbox >= BEBOP_PIPE_BATCH + BEBOP_PIPE_STAGES + 1, "a run's tasks plus the ring may each complete a sequence before the producer looks");
 
 struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of one (phase, wave) block from offset off
 

@@ -102,6 +102,13 @@ def test_draft_counts(K):
     full_check(cfg)
 
 
+def test_many_short_sequences_finish_in_quick_succession():
+    """Rows of one slice: every task completes a row, and a CTA's publisher completes sequences (accept scan,
+    draw set-up, the draw task mailed to its own producer) as fast as it publishes."""
+    cfg = G.Config("short", 3000, 1, 2040, "bf16", 2.0, True, 1.0, 1.0, seed=31)
+    full_check(cfg, sample=256)
+
+
 def test_all_draft_lengths_including_zero():
     cfg = G.Config("len", 10, 4, 4096, "f32", 2.0, False, 0.3, 1.0, seed=5)
     x = G.make_inputs(cfg, DEV)
