@@ -237,8 +237,14 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         if (wait) for (uint32_t i = 0; si.pad == 0 && i < kSpin; ++i) { __nanosleep(64); si = ld_cg(a.sinfo + b); }
         return si;
     };
+    SeqInfo seen; seen.n = 0; seen.draw_row = 0; seen.pad0 = 0; seen.pad = 0;     // the record `ready` last saw valid,
+    int seen_b = -1;                                                              // and whose it is
     auto ready = [&](int ph, int b, bool wait) {
-        if (ph == 2) return seq_info(b, wait).pad != 0;
+        if (ph != 2) return true;
+        if (seen_b == b) return true;
+        const SeqInfo si = seq_info(b, wait);
+        if (si.pad == 0) return false;
+        seen = si; seen_b = b;
         return true;
     };
     int it = 0, n_stream = 0, mb_head = 0;
@@ -340,7 +346,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 row0 = row_ptr(R, b, r);
             } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
-                const SeqInfo si = ld_cg(a.sinfo + b);
+                const SeqInfo si = seen_b == b ? seen : ld_cg(a.sinfo + b);
                 const int k = a.o.tv ? r : max(si.draw_row, 0);
                 d.r = k;
                 RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
@@ -350,7 +356,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 // overtaken that all the same, ask again)
                 if (k <= L) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
-                d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
+                d.c = __int_as_float(si.pad0);
                 const bool pair = k < L;
                 skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
                 // the sequence's second sweep: every half slice of the L row pairs, and of the bonus row if drawn from
@@ -478,7 +484,8 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
         if (a.o.row_status) a.o.row_status[b] = seq_st;
         a.stop[b] = fatal ? -1 : nn;
         // the record's mark makes it (and, through the row records it was computed from, the sequence) ready
-        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = 0; si.pad = 1;
+        // (pad0 carries c = log2(e) / tau of the sequence: the second sweep's producer need not divide again)
+        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = __float_as_int(ts.hi); si.pad = 1;
         st16(a.sinfo + b, si);
     }
 }
@@ -657,7 +664,6 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
     RowStat sp, sq;
     sp.inv_s = 0.0; sp.e = 0; sp.st = 0; sq = sp;
     if (lane == 0 && k >= 0) { sp = ld_cg(a.rstat + (int64_t)b * NR + k); if (pair) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k); }
-    const float tau = tau_of(R, b);
     if (lane < L && a.o.tv) {
         // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
         unsigned long long w = 0;
@@ -702,7 +708,7 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
             if (!room) atomicExch(a.wait_failed, 1);
             else {
                 DrawTask t;
-                t.tt = Tt; t.base = base; t.bound = (float)draw_bound(sumsq); t.c = temp_scale(tau).hi;
+                t.tt = Tt; t.base = base; t.bound = (float)draw_bound(sumsq); t.c = __int_as_float(si.pad0);
                 t.b = b; t.k = k; t.owner = owner; t.pair = pair ? 1 : 0;
                 t.P = row_scale(sp); t.Q = pair ? row_scale(sq) : no_row();
                 S.mbox[tail % kMbox] = t;
