@@ -617,21 +617,28 @@ __global__ void __launch_bounds__(kThreads) k_argmax(RowArgs a, float2* __restri
     float best = kNegInf;
     int bidx = INT_MAX;
     bool bad = false;
+    // branch-free over the vectors (so that several loads are on their way per thread): the best vector first,
+    // the index inside it from one more look at that vector
+    int bvec = -1;
+#pragma unroll 4
     for (int iv = begin + (int)threadIdx.x; iv < end; iv += kThreads) {
         float f[VEC];
         load_vec<DT>(row, iv, a.V, f);
         float vm = f[0];
 #pragma unroll
         for (int j = 1; j < VEC; ++j) vm = max_nan(vm, f[j]);
-        if (!(vm <= best)) {
-            if (!(vm < INFINITY)) bad = true;
-            else {
-                int jj = 0;
+        bad = bad || !(vm < INFINITY);                 // NaN or +inf
+        const bool better = vm > best;                 // strictly: the lowest vector wins a tie
+        best = better ? vm : best;
+        bvec = better ? iv : bvec;
+    }
+    if (bvec >= 0) {
+        float f[VEC];
+        load_vec<DT>(row, bvec, a.V, f);
+        int jj = 0;
 #pragma unroll
-                for (int j = VEC - 1; j >= 0; --j) if (f[j] == vm) jj = j;
-                best = vm; bidx = iv * VEC + jj;
-            }
-        }
+        for (int j = VEC - 1; j >= 0; --j) if (f[j] == best) jj = j;
+        bidx = bvec * VEC + jj;
     }
     if (bad) { best = __int_as_float(0x7fc00000); bidx = INT_MAX; }
 #pragma unroll
