@@ -204,6 +204,18 @@ def test_without_tv_same_tokens_on_a_large_vocabulary():
         assert torch.equal(a[k], b[k]), k
 
 
+@pytest.mark.parametrize("dtype,K,V", [("f32", 3, 1000), ("bf16", 32, 4096), ("bf16", 1, 70000)])
+def test_without_tv_matches_the_oracle(dtype, K, V):
+    """The shortened second sweep (tv = NULL) against the oracle directly: ragged lengths with L = 0, every K."""
+    cfg = G.Config("notv2", 12, K, V, dtype, 2.0, V > 5000, 1.0, 1.0, seed=23 + K)
+    x = G.make_inputs(cfg, DEV)
+    x["draft_len"] = torch.tensor([(i * 5) % (K + 1) for i in range(cfg.B)], dtype=torch.int32, device=DEV)
+    got = run_verify(x, want_tv=False)
+    torch.cuda.synchronize()
+    assert got["tv"] is None
+    compare_verify(got, oracle_on(x, None), cfg.dtype, None, context=cfg.name)
+
+
 def test_deterministic_and_stream_ordered():
     cfg = G.Config("det", 16, 3, 32768, "bf16", 3.0, True, 1.0, 1.0, seed=8)
     x = G.make_inputs(cfg, DEV)
