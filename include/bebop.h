@@ -119,7 +119,8 @@ bebop_status_t bebop_tv(
 
 /*
  * bebop_tv without a workspace argument (a convenience of this library; the paper has no
- * counterpart).  Same computation, same outputs and same errors as bebop_tv, with the per-slice
+ * counterpart).  Same definition, same outputs (to fp32 rounding: it always runs the split-row kernels,
+ * bebop_tv the pipelined kernel where the shape admits it) and same errors as bebop_tv, with the per-slice
  * partials of the sweep kept in a scratch array that is part of the library image
  * (BEBOP_TV_STATIC_SCRATCH_BYTES = 1 MiB, one copy per device).  The call allocates nothing and
  * frees nothing.

@@ -122,8 +122,16 @@ bebop_status_t bebop_tv(const void* target_logits, int64_t ld_target, const void
     if ((s = check_arch()) != BEBOP_OK) return s;
     RowArgs a = row_args(target_logits, ld_target, draft_logits, ld_draft, 1, 1, nullptr, temperature,
                          temperature_all, N, 1, V, dt, p);
-    cudaError_t e = general_tv(a, p, tv, s_aux, row_status, static_cast<char*>(workspace),
-                               static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSuccess;
+    bool launched = false;
+    if (g_path == 0 && pipe_supported(a)) {
+        // the pipelined kernel with row pairs in place of sequences: first sweep, second sweep, no draw
+        VerifyOut o{nullptr, nullptr, tv, nullptr, nullptr, row_status};
+        e = pipe_verify(a, p, nullptr, nullptr, nullptr, o, static_cast<char*>(workspace), stream, &launched, true, s_aux);
+    }
+    if (e == cudaSuccess && !launched)
+        e = general_tv(a, p, tv, s_aux, row_status, static_cast<char*>(workspace), stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
 

@@ -51,10 +51,11 @@ cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, c
                           cudaStream_t stream);
 
 // Pipelined kernel (bebop_pipe.cu): the wave schedule with a producer warp that stages every task's
-// logits in shared memory by bulk copies while the other warps compute; same contract.
+// logits in shared memory by bulk copies while the other warps compute; same contract.  With `tv_only` it is
+// bebop_tv: B row pairs (K = 1), o.tv and s_aux the outputs, no tokens, no uniforms, no draw.
 bool pipe_supported(const RowArgs& a);
 cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                        cudaStream_t stream, bool* launched);
+                        cudaStream_t stream, bool* launched, bool tv_only = false, float* s_aux = nullptr);
 
 }  // namespace bebop

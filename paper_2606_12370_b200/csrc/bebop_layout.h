@@ -22,7 +22,7 @@ struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 16)
     size_t off_p1done, off_p2done, off_xdone, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
-    size_t off_part, off_rstat, off_dpart, off_tvacc, off_sinfo, total;
+    size_t off_part, off_rstat, off_dpart, off_tvacc, off_sacc, off_sinfo, total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -61,6 +61,7 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.off_rstat = o;  o += align256(16 * (size_t)B * NR);
     w.off_dpart = o;  o += align256(16 * (size_t)B * 2 * w.T);
     w.off_tvacc = o;  o += align256(8 * (size_t)B * (K > 0 ? K : 1));
+    w.off_sacc = o;   o += align256(8 * (size_t)B * (K > 0 ? K : 1));
     w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.zero_bytes = o;
     w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);

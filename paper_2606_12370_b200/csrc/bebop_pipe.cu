@@ -191,13 +191,14 @@ __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinter
 // once per row.  Draw tasks have no tickets: the publisher warp of this CTA leaves one in the CTA's mailbox
 // when it has delivered the last partial of a sequence's second sweep, and the producer stages it ahead of
 // the next ticket.  Returns when the stop description has been handed to the consumers.
-template <int DT>
+template <int DT, bool TVO>
 __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsigned char* data) {
     const RowArgs& R = a.r;
     const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
     const int B = R.B;
     // (a caller that asks for no TV needs the second sweep over one row per sequence only: the one a token is drawn from)
-    const int c0 = NR * T, c2 = (a.o.tv ? K + 1 : 1) * T2;
+    // (and bebop_tv has the K row pairs and no bonus row)
+    const int c0 = NR * T, c2 = (TVO ? K : (a.o.tv ? K + 1 : 1)) * T2;
     const double inv_c0 = 1.0 / c0, inv_c2 = 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
     // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
@@ -342,7 +343,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 const bool is_target = r <= K;
                 const int k = is_target ? r : r - (K + 1);
                 d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
-                skip = is_target ? k > L : k >= L;
+                skip = is_target ? (TVO ? k >= L : k > L) : k >= L;     // (bebop_tv has no bonus row)
                 row0 = row_ptr(R, b, r);
             } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
@@ -354,11 +355,12 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 const int L = len_of(R, b);
                 // (the accept scan saw these row records before it set the sequence's mark; should a load have
                 // overtaken that all the same, ask again)
-                if (k <= L) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
+                const bool no_row_k = TVO && k >= L;      // bebop_tv has no bonus row: nothing was merged for it
+                if (k <= L && !no_row_k) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
                 d.c = __int_as_float(si.pad0);
                 const bool pair = k < L;
-                skip = k > L || si.n < 0 || (!pair && si.draw_row != L);
+                skip = k > L || si.n < 0 || (!pair && si.draw_row != L) || no_row_k;
                 // the sequence's second sweep: every half slice of the L row pairs, and of the bonus row if drawn from
                 d.need = T2 * (L + (si.draw_row == L ? 1 : 0));
                 if (!a.o.tv) d.need = T2;
@@ -422,7 +424,7 @@ __device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) 
     }
 }
 
-template <int DT>
+template <int DT, bool TVO>
 __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
@@ -432,8 +434,9 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     const TempScale ts = temp_scale(tau);
     // lane k owns draft position k (K <= 32): everything it needs is requested before anything is used
     const bool active = lane < L;
-    const int tk = active ? a.draft_tokens[(int64_t)b * K + lane] : 0;
-    const float u = active ? a.u_accept[(int64_t)b * K + lane] : 0.f;
+    const bool tvo = TVO;              // row pairs only: no tokens, no accept test, no bonus row
+    const int tk = (active && !tvo) ? a.draft_tokens[(int64_t)b * K + lane] : 0;
+    const float u = (active && !tvo) ? a.u_accept[(int64_t)b * K + lane] : 0.f;
     RowStat sp, sq, sb;
     sp.inv_s = 0.0; sp.e = E_EMPTY; sp.st = 0;
     sq = sp;
@@ -445,11 +448,11 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
         return x;
     };
     if (active) { sp = row(lane); sq = row(K + 1 + lane); }
-    sb = row(L);                                                       // bonus row (row L <= K: always merged)
+    if (tvo) { sb = sp; sb.st = 0; } else sb = row(L);                  // bonus row (row L <= K: always merged)
     int seq_st = ok ? 0 : ST_BAD_TEMP;
-    const bool tok_ok = tk >= 0 && tk < V;
+    const bool tok_ok = tvo || (tk >= 0 && tk < V);
     float zpx = 0.f, zqx = 0.f;
-    if (active && tok_ok) { zpx = load_one<DT>(row_ptr(R, b, lane), tk); zqx = load_one<DT>(row_ptr(R, b, K + 1 + lane), tk); }
+    if (active && tok_ok && !tvo) { zpx = load_one<DT>(row_ptr(R, b, lane), tk); zqx = load_one<DT>(row_ptr(R, b, K + 1 + lane), tk); }
     if (!seq_st && __ballot_sync(0xffffffffu, active && !tok_ok)) seq_st = ST_BAD_TOKEN;
     // the first bad row pair decides the status; rows after it do not count
     const int rs = active ? (sp.st | sq.st) : 0;
@@ -459,7 +462,7 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     if (!seq_st && badrows) seq_st = rs_first;
     double px = 0.0, qx = 0.0;
     bool acc = false;
-    if (active && !(seq_st & ST_FATAL) && lane < first_bad) {
+    if (active && !tvo && !(seq_st & ST_FATAL) && lane < first_bad) {
         const double cd = (double)ts.hi;
         px = exp2((double)zpx * cd - (double)sp.e) * sp.inv_s;
         qx = exp2((double)zqx * cd - (double)sq.e) * sq.inv_s;
@@ -471,21 +474,21 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
     const bool fatal = (seq_st & ST_FATAL) != 0;
     const int nn = fatal ? 0 : n;
     // outputs: lane q writes position q (position nn is filled by the draw)
-    for (int q = lane; q <= K; q += 32)
+    if (!tvo) for (int q = lane; q <= K; q += 32)
         if (fatal || q != nn) a.o.out_tokens[(int64_t)b * (K + 1) + q] = q < nn ? tk : -1;   // q < nn <= 32: q == lane
     if (lane < K) {
         const bool zero = fatal || lane >= L;
         if (a.o.p_draft) a.o.p_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)px;
         if (a.o.q_draft) a.o.q_draft[(int64_t)b * K + lane] = zero ? 0.f : (float)qx;
         if (zero && a.o.tv) a.o.tv[(int64_t)b * K + lane] = 0.f;
+        if (TVO && zero && a.s_aux) a.s_aux[(int64_t)b * K + lane] = 0.f;
     }
     if (lane == 0) {
-        a.o.accept_len[b] = nn;
+        if (!tvo) { a.o.accept_len[b] = nn; a.stop[b] = fatal ? -1 : nn; }
         if (a.o.row_status) a.o.row_status[b] = seq_st;
-        a.stop[b] = fatal ? -1 : nn;
         // the record's mark makes it (and, through the row records it was computed from, the sequence) ready
         // (pad0 carries c = log2(e) / tau of the sequence: the second sweep's producer need not divide again)
-        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = fatal ? -1 : nn; si.pad0 = __float_as_int(ts.hi); si.pad = 1;
+        SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = (fatal || tvo) ? -1 : nn; si.pad0 = __float_as_int(ts.hi); si.pad = 1;
         st16(a.sinfo + b, si);
     }
 }
@@ -566,7 +569,7 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
 // P2: TV partial of one half slice of a row pair; on the pair (or bonus row) a token is drawn from,
 // also the mass in double and the sum of squares.  Target row in the first half of the stage, draft
 // row in the second.
-template <int DT>
+template <int DT, bool TVO>
 __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
                                         int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / (2 * PC);
@@ -602,7 +605,24 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
     }
     float z0 = 0.f, z1 = 0.f, sqs = 0.f;
     double zd = 0.0;
-    if (!draw) {
+    if (TVO && a.sacc) {
+        // bebop_tv with the auxiliary sum: TV and S = sum of q over the tokens with q <= p (Eq. tv_grad)
+        float sx = 0.f;
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            float fp[VEC], fq[VEC];
+            unpack<DT>(rp[u], fp);
+            unpack<DT>(rq[u], fq);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float p = __fmul_rn(exp2_scaled(fp[i], c, SP.ef), SP.inv);
+                const float q = __fmul_rn(exp2_scaled(fq[i], c, SQ.ef), SQ.inv);
+                z0 += fmaxf(p - q, 0.f);
+                sx += q <= p ? q : 0.f;
+            }
+        }
+        zd = (double)warp_sum(sx);
+    } else if (!draw) {
 #pragma unroll
         for (int u = 0; u < NV; ++u) {
             float r[8];
@@ -625,7 +645,7 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
         }
     }
     const float z = warp_sum(z0 + z1);
-    if (draw) { zd = warp_sum(zd); sqs = warp_sum(sqs); }
+    if (draw && !(TVO && a.sacc)) { zd = warp_sum(zd); sqs = warp_sum(sqs); }
     if (lane == 0) { S.wf[stage][0][warp] = z; S.wd[stage][warp] = zd; S.wf[stage][1][warp] = sqs; }
     __syncwarp();
     if (lane == 0) mbar_arrive(&S.pdone[stage]);
@@ -652,6 +672,7 @@ __device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
 // sweep: TV of every draft position from the fixed-point sums, then the residual mass Z of the draw rows, the
 // target u * Z of the inverse CDF and the half slice that owns it.  The draw task goes into the CTA's mailbox:
 // the producer stages that half slice and the consumers find the token.
+template <bool TVO>
 __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, int b) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
@@ -675,6 +696,16 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         if ((int)(w & 0xffffull) < T2) atomicExch(a.wait_failed, 1);
         const float z = (float)((double)(w >> 16) * 9.094947017729282e-13);      // 2^-40
         a.o.tv[(int64_t)b * K + lane] = fminf(fmaxf(z, 0.f), 1.f);
+    }
+    if (TVO && lane < L && a.s_aux) {
+        unsigned long long w = 0;
+        for (uint32_t i = 0; i < kSpin; ++i) {
+            w = __ldcg(a.sacc + (int64_t)b * K + lane);
+            if ((int)(w & 0xffffull) >= T2) break;
+            __nanosleep(64);
+        }
+        if ((int)(w & 0xffffull) < T2) atomicExch(a.wait_failed, 1);
+        a.s_aux[(int64_t)b * K + lane] = (float)((double)(w >> 16) * 9.094947017729282e-13);
     }
     if (k < 0) return;
     // the half slices' masses: lanes fetch them in parallel, lane 0 scans them in slice order
@@ -823,7 +854,7 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
 // P1 -- the slice's (E, S) partial and the row's counter, whose last increment starts the merge of the
 // row, whose last merged row starts the accept scan of the sequence; P2 -- the TV part (and the
 // draw-row mass) and the sequence's counter.
-template <int DT>
+template <int DT, bool TVO>
 __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
@@ -872,10 +903,10 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
             }
             if (__shfl_sync(0xffffffffu, run_a, 0)) {
                 merge_row_warp(a, b, r);
-                // the last merged row of the sequence (2L+1 rows are in use) starts the accept scan
+                // the last merged row of the sequence (2L+1 rows are in use, 2L without a bonus row) starts the accept scan
                 int last_row = 0;
-                if (lane == 0) last_row = atomicAdd(&a.p1done[b], 1) == 2 * len_of(R, b);
-                if (__shfl_sync(0xffffffffu, last_row, 0)) accept_warp<DT>(a, b);
+                if (lane == 0) last_row = atomicAdd(&a.p1done[b], 1) == 2 * len_of(R, b) - (TVO ? 1 : 0);
+                if (__shfl_sync(0xffffffffu, last_row, 0)) accept_warp<DT, TVO>(a, b);
             }
         } else {
             float zz = 0.f, sq = 0.f; double tot = 0.0;
@@ -888,6 +919,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
                 // Fixed point with a count of one in the low bits of the same word: one relaxed add publishes value
                 // and count together, and integer sums do not depend on the order of arrival.
                 if (flags & 1) red_add_u64(a.tvacc + (int64_t)b * K + r, ((unsigned long long)__double2ll_rn((double)zz * kFixTv) << 16) | 1ull);
+                if (TVO && a.sacc) red_add_u64(a.sacc + (int64_t)b * K + r, ((unsigned long long)__double2ll_rn(tot * kFixTv) << 16) | 1ull);
                 if (flags & 2) {
                     unsigned long long* wd = a.dacc + ((int64_t)b * T2 + sl) * 2;
                     red_add_u64(wd, ((unsigned long long)__double2ll_rn(tot * kFixMass) << 4) | 1ull);
@@ -896,7 +928,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
                 // the sequence's last partial starts the set-up of its draw
                 run_d = atomicAdd(a.p2done + b, 1) == need - 1;
             }
-            if (__shfl_sync(0xffffffffu, run_d, 0)) draw_setup_warp(a, S, b);
+            if (__shfl_sync(0xffffffffu, run_d, 0)) draw_setup_warp<TVO>(a, S, b);
         }
         // the producer stays until every streaming task has been dealt with here (mailbox entries come first)
         __syncwarp();
@@ -906,7 +938,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
 
 }  // namespace
 
-template <int DT>
+template <int DT, bool TVO>
 __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ WaveArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* data = smem;
@@ -923,8 +955,8 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     }
     __syncthreads();
     if (tid >= PC) {
-        if (tid == PC) producer<DT>(a, S, data);
-        else if (tid >= PC + 32) publisher<DT>(a, S);
+        if (tid == PC) producer<DT, TVO>(a, S, data);
+        else if (tid >= PC + 32) publisher<DT, TVO>(a, S);
         return;
     }
     const int lane = tid & 31;
@@ -937,7 +969,7 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (tid == 0) PLOG(2, it);
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
         if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
-        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
+        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT, TVO>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
         else {
             if (tid == 0) PTLOG(2);
             pipe_d<DT>(a, S, d, sd);
@@ -955,18 +987,18 @@ namespace {
 
 constexpr size_t kPipeSmem = (size_t)NST * STAGE_BYTES + sizeof(PipeShared);
 
-template <int DT>
+template <int DT, bool TVO>
 int pipe_grid() {
     static int cached[64] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
-    if (cudaFuncSetAttribute(k_pipe<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_pipe<DT, TVO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
     int per_sm = 0, sms = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pipe<DT>, PT, kPipeSmem) != cudaSuccess) per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pipe<DT, TVO>, PT, kPipeSmem) != cudaSuccess) per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaGetLastError();
     const int n = per_sm * sms;
@@ -986,9 +1018,10 @@ bool pipe_supported(const RowArgs& a) {
 
 cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
-                        cudaStream_t stream, bool* launched) {
+                        cudaStream_t stream, bool* launched, bool tv_only, float* s_aux) {
     *launched = false;
-    const int grid_max = a.dt == 0 ? pipe_grid<0>() : pipe_grid<1>();
+    const int grid_max = tv_only ? (a.dt == 0 ? pipe_grid<0, true>() : pipe_grid<1, true>())
+                                 : (a.dt == 0 ? pipe_grid<0, false>() : pipe_grid<1, false>());
     if (grid_max < 1) return cudaSuccess;
     const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
     WaveArgs wa;
@@ -1007,11 +1040,14 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.dacc = reinterpret_cast<unsigned long long*>(w + wp.off_dpart);
     wa.tvacc = reinterpret_cast<unsigned long long*>(w + wp.off_tvacc);
     wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
+    wa.tv_only = tv_only ? 1 : 0;
+    wa.s_aux = tv_only ? s_aux : nullptr;
+    wa.sacc = (tv_only && s_aux) ? reinterpret_cast<unsigned long long*>(w + wp.off_sacc) : nullptr;
     wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
     {
         const long long NR = 2 * a.K + 1;
-        const long long total = (long long)a.B * (NR * wp.T + (long long)(o.tv ? a.K + 1 : 1) * 2 * wp.T);
+        const long long total = (long long)a.B * (NR * wp.T + (long long)(tv_only ? a.K : (o.tv ? a.K + 1 : 1)) * 2 * wp.T);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
         // Distance of the second sweep behind the first, in sequences.  The default is the whole batch (two full
@@ -1031,8 +1067,13 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     if (e != cudaSuccess) return e;
     const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
     if (g_ev_start) cudaEventRecord(g_ev_start, stream);
-    if (a.dt == 0) k_pipe<0><<<grid, PT, kPipeSmem, stream>>>(wa);
-    else k_pipe<1><<<grid, PT, kPipeSmem, stream>>>(wa);
+    if (tv_only) {
+        if (a.dt == 0) k_pipe<0, true><<<grid, PT, kPipeSmem, stream>>>(wa);
+        else k_pipe<1, true><<<grid, PT, kPipeSmem, stream>>>(wa);
+    } else {
+        if (a.dt == 0) k_pipe<0, false><<<grid, PT, kPipeSmem, stream>>>(wa);
+        else k_pipe<1, false><<<grid, PT, kPipeSmem, stream>>>(wa);
+    }
     e = cudaGetLastError();
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;

@@ -55,6 +55,9 @@ struct WaveArgs {
     unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
     int ntickets, lag;               // distance (sequences) of P2 behind P1
+    int tv_only;                     // bebop_tv: row pairs only (no bonus row, no accept test, no draw)
+    float* s_aux;                    // tv_only: [B] sum of q over the tokens with q <= p, or nullptr
+    unsigned long long* sacc;        // [B][K] that sum in 2^-40 units << 16 | parts added
     long long* trace;
     int T, slice_vecs;
 };

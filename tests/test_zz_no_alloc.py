@@ -24,12 +24,17 @@ def test_static_equals_workspace_two_calls_in_a_row(dtype, N, V):
             tgt[1, 7:] = float("-inf")          # masked vocabulary
             drf[2, :] = tgt[2, :]               # identical rows: TV exactly 0
             tgt[3, 5] = float("nan")            # status bit
+        P.bebop_debug_force_general_path(1)     # bebop_tv through the same split-row kernels: bit for bit
         want = P.bebop_tv(tgt, drf, temperature=tau)
+        P.bebop_debug_force_general_path(0)     # and through the pipelined kernel: to rounding
+        fast = P.bebop_tv(tgt, drf, temperature=tau)
         got = P.bebop_tv_static(tgt, drf, temperature=tau)
         torch.cuda.synchronize()
-        assert torch.equal(got["row_status"], want["row_status"])
+        assert torch.equal(got["row_status"], want["row_status"]) and torch.equal(got["row_status"], fast["row_status"])
         assert torch.equal(got["tv"].view(torch.int32), want["tv"].view(torch.int32))          # bit for bit
         assert torch.equal(got["s_aux"].view(torch.int32), want["s_aux"].view(torch.int32))
+        assert float((got["tv"] - fast["tv"]).abs().max()) <= 1e-5
+        assert float((got["s_aux"] - fast["s_aux"]).abs().max()) <= 1e-5
         if call == 1:
             assert float(got["tv"][2]) == 0.0 and int(got["row_status"][3]) & 1
 
