@@ -150,8 +150,13 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
     if ((s = check_arch()) != BEBOP_OK) return s;
     RowArgs a = row_args(target_logits, ld_target, nullptr, 0, K + 1, K, draft_len, nullptr, 1.f, B, K,
                          V, dt, p);
-    cudaError_t e = general_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status,
-                                   static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSuccess;
+    bool launched = false;
+    if (g_path == 0 && pipe_supported(a))
+        e = pipe_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream, &launched);
+    if (e == cudaSuccess && !launched)
+        e = general_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
 

@@ -58,4 +58,9 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched, bool tv_only = false, float* s_aux = nullptr);
 
+// The greedy mode through the pipelined kernel: one sweep over the target rows (maximum and lowest index per
+// slice), then a small kernel that merges the slices and runs the argmax match.
+cudaError_t pipe_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_tokens, int32_t* accept_len,
+                        int32_t* out_tokens, int32_t* row_status, char* ws, cudaStream_t stream, bool* launched);
+
 }  // namespace bebop

@@ -57,6 +57,9 @@ namespace {
 #ifndef BEBOP_PIPE_CTAS
 #define BEBOP_PIPE_CTAS 3
 #endif
+// what the kernel is compiled for: bebop_verify; bebop_tv (row pairs, no accept test, no draw); the greedy mode
+// (one sweep over the target rows for their argmax)
+constexpr int kModeVerify = 0, kModeTv = 1, kModeGreedy = 2;
 constexpr int NST = BEBOP_PIPE_STAGES;            // stages of the ring
 constexpr int PIPE_CTAS = BEBOP_PIPE_CTAS;        // CTAs per SM the kernel is built for
 constexpr int PC = WT;                            // consumer threads (8 warps); thread PC is the producer
@@ -191,15 +194,17 @@ __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinter
 // once per row.  Draw tasks have no tickets: the publisher warp of this CTA leaves one in the CTA's mailbox
 // when it has delivered the last partial of a sequence's second sweep, and the producer stages it ahead of
 // the next ticket.  Returns when the stop description has been handed to the consumers.
-template <int DT, bool TVO>
+template <int DT, int MODE>
 __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsigned char* data) {
+    constexpr bool TVO = MODE == kModeTv, GRD = MODE == kModeGreedy;
     const RowArgs& R = a.r;
     const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
     const int B = R.B;
     // (a caller that asks for no TV needs the second sweep over one row per sequence only: the one a token is drawn from)
     // (and bebop_tv has the K row pairs and no bonus row)
-    const int c0 = NR * T, c2 = (TVO ? K : (a.o.tv ? K + 1 : 1)) * T2;
-    const double inv_c0 = 1.0 / c0, inv_c2 = 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
+    // (the greedy mode sweeps the K + 1 target rows once)
+    const int c0 = (GRD ? K + 1 : NR) * T, c2 = GRD ? 0 : (TVO ? K : (a.o.tv ? K + 1 : 1)) * T2;
+    const double inv_c0 = 1.0 / c0, inv_c2 = GRD ? 0.0 : 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
     // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
     // exists).  With W = B (the default) that is all of P1, then all of P2: two full sweeps, sequences ascending,
@@ -217,7 +222,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         if (W >= B && f_next <= t) {
             // two full sweeps: the block follows from one division (a CTA's next tickets are some thirty blocks
             // on: stepping there one block at a time was most of what the producer did between two runs)
-            blk = t < B * c0 ? div_by(t, c0, inv_c0) : B + div_by(t - B * c0, c2, inv_c2);
+            blk = (GRD || t < B * c0) ? div_by(t, c0, inv_c0) : B + div_by(t - B * c0, c2, inv_c2);
             f_here = before(blk); f_next = before(blk + 1);
         }
         while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
@@ -342,7 +347,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 const int L = len_of(R, b);
                 const bool is_target = r <= K;
                 const int k = is_target ? r : r - (K + 1);
-                d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi;
+                if (!GRD) { d.tau = tau_of(R, b); d.c = temp_scale(d.tau).hi; }
                 skip = is_target ? (TVO ? k >= L : k > L) : k >= L;     // (bebop_tv has no bonus row)
                 row0 = row_ptr(R, b, r);
             } else {
@@ -562,6 +567,53 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
     float mw = ord2f(redux_max(f2ord(bad ? -INFINITY : m)));
     if (anybad) mw = __int_as_float(0x7fc00000);
     if (lane == 0) { S.wf[stage][0][warp] = st; S.wi[stage][warp] = Ew; S.wf[stage][1][warp] = mw; }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&S.pdone[stage]);
+}
+
+// Greedy mode: maximum and lowest index of the maximum over one slice of a target row (no exponentials).
+template <int DT>
+__device__ __forceinline__ void pipe_g(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+                                       int stage) {
+    constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
+    const RowArgs& R = a.r;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nv = d.nv;
+    uint4 raw[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        const int v = tid + u * PC;
+        raw[u] = neg_inf_vec<DT>();
+        if (v < nv) raw[u] = lds16(data + (size_t)v * 16);
+    }
+    if ((d.v0 + nv) * VEC > R.V) {               // the row's last vector is in this slice and is partial
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int gbase = (d.v0 + tid + u * PC) * VEC;
+            if (tid + u * PC < nv && gbase + VEC > R.V) mask_tail<DT>(raw[u], R.V - gbase);
+        }
+    }
+    float m = vec_max<DT>(raw[0]);
+#pragma unroll
+    for (int u = 1; u < NV; ++u) m = max_nan(m, vec_max<DT>(raw[u]));
+    if (!(m < INFINITY)) m = __int_as_float(0x7fc00000);      // NaN or +inf poisons the row
+    // the thread's lowest token with that value (its vectors ascend with u)
+    int idx = INT_MAX;
+    if (m == m && m > -INFINITY) {
+#pragma unroll
+        for (int u = NV - 1; u >= 0; --u) {
+            float f[VEC];
+            unpack<DT>(raw[u], f);
+#pragma unroll
+            for (int j = VEC - 1; j >= 0; --j) if (f[j] == m) idx = (d.v0 + tid + u * PC) * VEC + j;
+        }
+    }
+    // warp: the maximum (NaN sorts above +inf), then the lowest index among the lanes that hold it
+    const int om = f2ord(m);
+    const int ow = redux_max(om);
+    int iw;
+    { const int mine = om == ow ? idx : INT_MAX; asm volatile("redux.sync.min.s32 %0, %1, 0xffffffff;" : "=r"(iw) : "r"(mine)); }
+    if (lane == 0) { S.wi[stage][warp] = ow; S.wf[stage][0][warp] = __int_as_float(iw); }
     __syncwarp();
     if (lane == 0) mbar_arrive(&S.pdone[stage]);
 }
@@ -854,8 +906,9 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
 // P1 -- the slice's (E, S) partial and the row's counter, whose last increment starts the merge of the
 // row, whose last merged row starts the accept scan of the sequence; P2 -- the TV part (and the
 // draw-row mass) and the sequence's counter.
-template <int DT, bool TVO>
+template <int DT, int MODE>
 __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
+    constexpr bool TVO = MODE == kModeTv, GRD = MODE == kModeGreedy;
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, T2 = 2 * a.T;
@@ -883,7 +936,20 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
         const int ii = S.wi[stage][w];
         __syncwarp();
         if (lane == 0) mbar_arrive(&S.empty[stage]);
-        if (phase == 0) {
+        if (GRD) {
+            // lanes 0..7 hold the warps' (maximum, lowest index): the slice's record, read by the kernel that finishes
+            const int iw = __float_as_int(f0);
+            int om = ii;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) om = max(om, __shfl_xor_sync(0xffffffffu, om, o));
+            int im = ii == om ? iw : INT_MAX;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) im = min(im, __shfl_xor_sync(0xffffffffu, im, o));
+            if (lane == 0) {
+                P1Part p; p.s = (double)im; p.e = 1; p.m = ord2f(om);
+                st16(a.part + ((int64_t)b * (2 * K + 1) + r) * a.T + sl, p);
+            }
+        } else if (phase == 0) {
             // lanes 0..7 hold the warps' (sum, exponent, max); merge in warp order
             const int Ec = max(max(max(__shfl_sync(0xffffffffu, ii, 0), __shfl_sync(0xffffffffu, ii, 1)),
                                    max(__shfl_sync(0xffffffffu, ii, 2), __shfl_sync(0xffffffffu, ii, 3))),
@@ -938,7 +1004,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
 
 }  // namespace
 
-template <int DT, bool TVO>
+template <int DT, int MODE>
 __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ WaveArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* data = smem;
@@ -955,8 +1021,8 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     }
     __syncthreads();
     if (tid >= PC) {
-        if (tid == PC) producer<DT, TVO>(a, S, data);
-        else if (tid >= PC + 32) publisher<DT, TVO>(a, S);
+        if (tid == PC) producer<DT, MODE>(a, S, data);
+        else if (tid >= PC + 32) publisher<DT, MODE>(a, S);
         return;
     }
     const int lane = tid & 31;
@@ -968,8 +1034,9 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         if (d.phase < 0) break;
         if (tid == 0) PLOG(2, it);
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
-        if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
-        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT, TVO>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
+        if (MODE == kModeGreedy) pipe_g<DT>(a, S, d, sd, stage);
+        else if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
+        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT, MODE == kModeTv>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
         else {
             if (tid == 0) PTLOG(2);
             pipe_d<DT>(a, S, d, sd);
@@ -987,18 +1054,18 @@ namespace {
 
 constexpr size_t kPipeSmem = (size_t)NST * STAGE_BYTES + sizeof(PipeShared);
 
-template <int DT, bool TVO>
+template <int DT, int MODE>
 int pipe_grid() {
     static int cached[64] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
-    if (cudaFuncSetAttribute(k_pipe<DT, TVO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_pipe<DT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
     int per_sm = 0, sms = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pipe<DT, TVO>, PT, kPipeSmem) != cudaSuccess) per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pipe<DT, MODE>, PT, kPipeSmem) != cudaSuccess) per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaGetLastError();
     const int n = per_sm * sms;
@@ -1020,8 +1087,8 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched, bool tv_only, float* s_aux) {
     *launched = false;
-    const int grid_max = tv_only ? (a.dt == 0 ? pipe_grid<0, true>() : pipe_grid<1, true>())
-                                 : (a.dt == 0 ? pipe_grid<0, false>() : pipe_grid<1, false>());
+    const int grid_max = tv_only ? (a.dt == 0 ? pipe_grid<0, kModeTv>() : pipe_grid<1, kModeTv>())
+                                 : (a.dt == 0 ? pipe_grid<0, kModeVerify>() : pipe_grid<1, kModeVerify>());
     if (grid_max < 1) return cudaSuccess;
     const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
     WaveArgs wa;
@@ -1068,17 +1135,102 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
     if (g_ev_start) cudaEventRecord(g_ev_start, stream);
     if (tv_only) {
-        if (a.dt == 0) k_pipe<0, true><<<grid, PT, kPipeSmem, stream>>>(wa);
-        else k_pipe<1, true><<<grid, PT, kPipeSmem, stream>>>(wa);
+        if (a.dt == 0) k_pipe<0, kModeTv><<<grid, PT, kPipeSmem, stream>>>(wa);
+        else k_pipe<1, kModeTv><<<grid, PT, kPipeSmem, stream>>>(wa);
     } else {
-        if (a.dt == 0) k_pipe<0, false><<<grid, PT, kPipeSmem, stream>>>(wa);
-        else k_pipe<1, false><<<grid, PT, kPipeSmem, stream>>>(wa);
+        if (a.dt == 0) k_pipe<0, kModeVerify><<<grid, PT, kPipeSmem, stream>>>(wa);
+        else k_pipe<1, kModeVerify><<<grid, PT, kPipeSmem, stream>>>(wa);
     }
     e = cudaGetLastError();
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;
     *launched = true;
     return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, wa.wait_failed, w, wp, stream);
+}
+
+// ------------------------------------------------------------------ greedy mode
+namespace {
+
+// One warp per sequence, behind the sweep: lane k merges the slice records of target row k (maximum, lowest
+// index), then the argmax match x_k == g_k runs down the drafts; the argmax of the stop position is emitted.
+__global__ void __launch_bounds__(128) k_greedy_finish(WaveArgs a, int32_t* __restrict__ accept_len,
+                                                        int32_t* __restrict__ out_tokens, int32_t* __restrict__ row_status) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // programmatic dependent of the sweep
+    const RowArgs& R = a.r;
+    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= R.B) return;
+    const int K = R.K, L = len_of(R, b), NR = 2 * K + 1;
+    int st = *a.wait_failed ? ST_WAIT : 0;
+    const int tok = lane < L ? a.draft_tokens[(int64_t)b * K + lane] : -1;
+    if (lane < L && (tok < 0 || tok >= R.V)) st |= ST_BAD_TOKEN;
+    // lanes 0..L merge the target rows 0..L (two rounds when L + 1 > 32)
+    int g = -1, g_bonus = -1;
+    for (int round = 0; round < 2; ++round) {
+        const int k = round == 0 ? lane : 32 + lane;
+        if (k <= L && k <= K) {
+            const P1Part* pp = a.part + ((int64_t)b * NR + k) * a.T;
+            float best = -INFINITY; int bidx = INT_MAX;
+            for (int s = 0; s < a.T; ++s) {
+                const P1Part rec = pp[s];
+                if (rec.m != rec.m) { best = rec.m; break; }
+                if (rec.m > best) { best = rec.m; bidx = (int)rec.s; }        // slices ascend: the lowest index wins a tie
+            }
+            if (best != best) st |= ST_NONFINITE;
+            else if (best == -INFINITY) st |= ST_EMPTY;
+            if (round == 0) g = bidx; else g_bonus = bidx;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) st |= __shfl_xor_sync(0xffffffffu, st, off);
+    if (st & ST_FATAL) {
+        if (lane <= K) out_tokens[(int64_t)b * (K + 1) + lane] = -1;
+        if (K == 32 && lane == 0) out_tokens[(int64_t)b * (K + 1) + 32] = -1;
+        if (lane == 0) { accept_len[b] = 0; if (row_status) row_status[b] = st; }
+        return;
+    }
+    const unsigned mis = __ballot_sync(0xffffffffu, lane < L && tok != g);
+    const int n = mis ? (__ffs(mis) - 1) : L;
+    const int y = n < 32 ? __shfl_sync(0xffffffffu, g, n & 31) : __shfl_sync(0xffffffffu, g_bonus, 0);
+    if (lane <= K && lane < 32) out_tokens[(int64_t)b * (K + 1) + lane] = lane < n ? tok : (lane == n ? y : -1);
+    if (K == 32 && lane == 0) out_tokens[(int64_t)b * (K + 1) + 32] = (n == 32) ? y : -1;
+    if (lane == 0) { accept_len[b] = n; if (row_status) row_status[b] = st; }
+}
+
+}  // namespace
+
+cudaError_t pipe_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_tokens, int32_t* accept_len,
+                        int32_t* out_tokens, int32_t* row_status, char* ws, cudaStream_t stream, bool* launched) {
+    *launched = false;
+    const int grid_max = a.dt == 0 ? pipe_grid<0, kModeGreedy>() : pipe_grid<1, kModeGreedy>();
+    if (grid_max < 1) return cudaSuccess;
+    const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
+    const long long total = (long long)a.B * (a.K + 1) * wp.T;
+    if (total > 0x7fff0000LL) return cudaSuccess;
+    char* w = ws + p.off_wave;
+    WaveArgs wa = {};
+    wa.r = a; wa.draft_tokens = draft_tokens;
+    wa.ticket = reinterpret_cast<int*>(w);
+    wa.wait_failed = wa.ticket + 1;
+    wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
+    wa.trace = g_wave_trace;
+    wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
+    wa.ntickets = (int)total; wa.lag = a.B;
+    cudaError_t e = cudaMemsetAsync(w, 0, 256, stream);       // ticket counter and wait flag
+    if (e != cudaSuccess) return e;
+    const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;
+    if (a.dt == 0) k_pipe<0, kModeGreedy><<<grid, PT, kPipeSmem, stream>>>(wa);
+    else k_pipe<1, kModeGreedy><<<grid, PT, kPipeSmem, stream>>>(wa);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    *launched = true;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((a.B + 3) / 4); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_greedy_finish, wa, accept_len, out_tokens, row_status);
 }
 
 }  // namespace bebop
