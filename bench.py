@@ -268,6 +268,25 @@ def run_ours(args):
     barrier()
     notv_ms = n0.elapsed_time(n1) / notv_steps
 
+    # the two other entry points on the same logits (reported beside the headline, not part of it)
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(n):
+            fn()
+        a1.record()
+        barrier()
+        return a0.elapsed_time(a1) / n
+
+    other_steps = max(1, min(steps, 50))
+    tv_t = x["target"][:, :K].reshape(B * K, V)
+    tv_d = x["draft"].reshape(B * K, V)
+    tv_ms = timed(lambda: P.bebop_tv(tv_t, tv_d, temperature_all=1.0), other_steps)
+    gr_ms = timed(lambda: P.bebop_greedy_verify(x["target"], x["draft_tokens"]), other_steps)
+
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
     e2e_steps = 0 if args.no_e2e else max(1, min(steps, 10))
     host = {k: x[k].cpu().pin_memory() for k in ("target", "draft", "draft_tokens", "u_accept", "u_final")}
@@ -297,7 +316,7 @@ def run_ours(args):
 
     # max over ranks
     from paper_2606_12370_b200.shard import max_over_ranks
-    ms, e2e_s, notv_ms = max_over_ranks([ms, e2e_s, notv_ms], dist, dev)
+    ms, e2e_s, notv_ms, tv_ms, gr_ms = max_over_ranks([ms, e2e_s, notv_ms, tv_ms, gr_ms], dist, dev)
     sampler.stop()
 
     if rank == 0:
@@ -319,6 +338,11 @@ def run_ours(args):
             "e2e": {"value": world * positions / e2e_s, "unit": "positions/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3},
             "gpu_launches": steps * launches_per_call,
+            "other_entry_points": {
+                "bebop_tv": {"ms_per_call": tv_ms, "row_pairs": world * B * K, "steps": other_steps,
+                             "algorithmic_gbs": world * B * K * 2 * V * es / (tv_ms * 1e-3) / 1e9},
+                "bebop_greedy_verify": {"ms_per_call": gr_ms, "steps": other_steps,
+                                        "algorithmic_gbs": world * B * (K + 1) * V * es / (gr_ms * 1e-3) / 1e9}},
             "without_tv": {"value": world * positions / (notv_ms * 1e-3), "unit": "positions/s", "ms_per_step": notv_ms,
                            "steps": notv_steps, "note": "same call with tv = NULL; not the headline"},
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,

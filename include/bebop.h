@@ -160,8 +160,8 @@ bebop_status_t bebop_greedy_verify(
 
 /*
  * Test and measurement hooks (no counterpart in the paper).
- * bebop_debug_force_general_path(1) makes bebop_verify use the split-row general
- * kernels even for shapes the pipelined kernel takes (process-wide switch; 0 restores).
+ * bebop_debug_force_general_path(1) makes bebop_verify, bebop_tv and bebop_greedy_verify use the
+ * split-row general kernels even for shapes the pipelined kernel takes (process-wide switch; 0 restores).
  * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
  * shape, of an int32 that after a bebop_verify call holds the number of sequences
  * whose draw was re-done by the fp64 kernels.
