@@ -45,10 +45,13 @@ void wave_set_trace(long long* p);                            // trace buffer of
 void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the main kernel of the next calls (nullptr: off)
 
 // fp64 re-draw of the sequences a kernel listed (bebop_redraw.cu); `w` is the wave workspace laid out by `wp`.
-// It also turns a device-side wait that gave up (`wait_failed`) into status bit ST_WAIT of every row.
-cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const int* fb_count,
-                          const FbRec* fb_list, const int* wait_failed, char* w, const WavePlan& wp,
-                          cudaStream_t stream);
+// Launched behind the pipelined kernel, it follows the list while that kernel still runs: the low half of
+// `fb_count` is the number of listed sequences so far, the high half the number of sequences whose draw is
+// decided, `expect` of them in all.  It also turns a device-side wait that gave up (`wait_failed`) into status
+// bit ST_WAIT of every row.
+cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const unsigned long long* fb_count,
+                          const FbRec* fb_list, int expect, int* wait_failed, char* w,
+                          const WavePlan& wp, cudaStream_t stream);
 
 // Pipelined kernel (bebop_pipe.cu): the wave schedule with a producer warp that stages every task's
 // logits in shared memory by bulk copies while the other warps compute; same contract.  With `tv_only` it is

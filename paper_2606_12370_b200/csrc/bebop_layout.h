@@ -13,14 +13,19 @@ namespace bebop {
 constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
 // A sequence whose draw goes to the fp64 re-draw: all the re-draw kernels need to find its rows.
 struct alignas(16) FbRec {
-    int b;                              // sequence
+    int b1;                             // sequence + 1 (0: the record is not written yet)
     int kp;                             // 2 * draw row + (1 if the row is a residual of a target / draft pair)
     int ep, eq;                         // reference exponents of the target row and of the draft row
 };
-constexpr size_t kFbCountOffset = 128;   // int: sequences listed for the fp64 re-draw, inside the zeroed head of the workspace
+#ifndef BEBOP_REDRAW_CUT
+#define BEBOP_REDRAW_CUT 4
+#endif
+constexpr int kRedrawCut = BEBOP_REDRAW_CUT;   // the fp64 re-draw cuts every row slice into so many work items
+constexpr size_t kFbCountOffset = 128;   // 8 bytes inside the zeroed head of the workspace: low int, sequences listed for the fp64
+                                         // re-draw; high int, sequences whose draw is decided
 struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 16)
-    size_t off_p1done, off_p2done, off_xdone, off_rowcnt, zero_bytes;
+    size_t off_p1done, off_p2done, off_xdone, off_xsdone, off_fbrec, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
     size_t off_part, off_rstat, off_dpart, off_tvacc, off_sacc, off_sinfo, total;
 };
@@ -39,7 +44,6 @@ struct Plan {
     size_t off_dstats;  // double2[B][2][nsplit_d]       (m, S) partials, fp64
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
-    size_t off_fb;      // 16-byte records [B]: the sequences whose draw goes to fp64
     size_t off_wave;    // workspace of the pipelined kernel
     size_t total;
 };
@@ -55,6 +59,8 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per sequence: rows merged
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
+    w.off_xsdone = o; o += align256(sizeof(int) * (size_t)B);
+    w.off_fbrec = o;  o += align256(16 * (size_t)B);          // records of the sequences whose draw goes to fp64
     w.off_rowcnt = o; o += align256(sizeof(int) * (size_t)B * NR);
     // records that readers validate by a mark inside them, and sums that start from zero
     w.off_part = o;   o += align256(16 * (size_t)B * NR * w.T);
@@ -64,8 +70,8 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     w.off_sacc = o;   o += align256(8 * (size_t)B * (K > 0 ? K : 1));
     w.off_sinfo = o;  o += align256(16 * (size_t)B);
     w.zero_bytes = o;
-    w.off_xsum = o;   o += align256(16 * (size_t)B * 4 * w.T);
-    w.off_xmass = o;  o += align256(8 * (size_t)B * 4 * w.T * 8);
+    w.off_xsum = o;   o += align256(16 * (size_t)B * kRedrawCut * w.T);
+    w.off_xmass = o;  o += align256(8 * (size_t)B * kRedrawCut * w.T * 8);
     w.total = o;
     return w;
 }
@@ -96,7 +102,6 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dstats = o; o = align256(o + sizeof(double) * 2 * (size_t)B * 2 * nsd);
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
-    p.off_fb = o;     o = align256(o + 16 * (size_t)B);
     {
         p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
     }

@@ -495,6 +495,7 @@ __device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
         // (pad0 carries c = log2(e) / tau of the sequence: the second sweep's producer need not divide again)
         SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = (fatal || tvo) ? -1 : nn; si.pad0 = __float_as_int(ts.hi); si.pad = 1;
         st16(a.sinfo + b, si);
+        if (fatal && !tvo) draw_decided(a.fb_count);     // no draw will come
     }
 }
 
@@ -777,8 +778,8 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         if (owner < 0) {
             // no half slice owns the target (no residual mass, or u = 0): the fp64 re-draw decides
             FbRec rec;
-            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0); rec.ep = sp.e; rec.eq = pair ? sq.e : 0;
-            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
+            rec.b1 = b + 1; rec.kp = 2 * k + (pair ? 1 : 0); rec.ep = sp.e; rec.eq = pair ? sq.e : 0;
+            st16(a.fb_list + draw_listed(a.fb_count), rec);
         } else {
             // the mailbox has room for more draws than this CTA's unpublished tasks can bring; should it be full
             // all the same, wait (bounded) for the producer
@@ -889,13 +890,13 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
     if (tid == 0) {
         int y = -1, cnt = 0;
         for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
-        if (cnt == 1 && y >= 0) a.o.out_tokens[(int64_t)b * (K + 1) + k] = y;
+        if (cnt == 1 && y >= 0) { a.o.out_tokens[(int64_t)b * (K + 1) + k] = y; draw_decided(a.fb_count); }
         else {
             FbRec rec;
-            rec.b = b; rec.kp = 2 * k + (pair ? 1 : 0);
+            rec.b1 = b + 1; rec.kp = 2 * k + (pair ? 1 : 0);
             rec.ep = ld_cg(a.rstat + (int64_t)b * NR + k).e;
             rec.eq = pair ? ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k).e : 0;
-            st16(a.fb_list + atomicAdd(a.fb_count, 1), rec);
+            st16(a.fb_list + draw_listed(a.fb_count), rec);
         }
     }
 }
@@ -1010,8 +1011,8 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     unsigned char* data = smem;
     PipeShared& S = *reinterpret_cast<PipeShared*>(smem + (size_t)NST * STAGE_BYTES);
     const int tid = threadIdx.x;
-    // the re-draw kernel behind this one may be scheduled as CTAs of this one leave; it waits for this grid's
-    // completion before it reads anything (programmatic dependent launch)
+    // the re-draw kernel behind this one may be scheduled as CTAs of this one leave (programmatic dependent
+    // launch); it follows the list of sequences as it grows (`fb_count` tells it when the list is complete)
     if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) PTLOG(0);
     if (tid == 0) {
@@ -1095,8 +1096,8 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.r = a; wa.draft_tokens = draft_tokens; wa.u_accept = u_accept; wa.u_final = u_final; wa.o = o;
     wa.stop = reinterpret_cast<int*>(ws + p.off_stop);
     char* w = ws + p.off_wave;
-    wa.fb_count = reinterpret_cast<int*>(w + kFbCountOffset);
-    wa.fb_list = reinterpret_cast<FbRec*>(ws + p.off_fb);
+    wa.fb_count = reinterpret_cast<unsigned long long*>(w + kFbCountOffset);
+    wa.fb_list = reinterpret_cast<FbRec*>(w + wp.off_fbrec);
     wa.ticket = reinterpret_cast<int*>(w);
     wa.wait_failed = wa.ticket + 1;
     wa.p1done = reinterpret_cast<int*>(w + wp.off_p1done);
@@ -1145,7 +1146,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;
     *launched = true;
-    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, wa.wait_failed, w, wp, stream);
+    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, tv_only ? 0 : a.B, wa.wait_failed, w, wp, stream);
 }
 
 // ------------------------------------------------------------------ greedy mode

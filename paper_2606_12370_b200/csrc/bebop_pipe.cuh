@@ -41,8 +41,9 @@ struct WaveArgs {
     const float* u_final;
     VerifyOut o;
     int* stop;
-    int* fb_count;        // [1] sequences listed for the fp64 re-draw (zeroed with the workspace)
-    FbRec* fb_list;       // [B]
+    unsigned long long* fb_count;   // [1] low half: sequences listed for the fp64 re-draw; high half: sequences whose
+                                    // draw is decided (token written, listed, or none to come); zeroed with the workspace
+    FbRec* fb_list;       // [B] (zeroed with the workspace: a record is valid once its b1 is non-zero)
     // workspace
     int* ticket;          // [1]
     int* wait_failed;     // [1]
@@ -70,6 +71,14 @@ __device__ __forceinline__ int len_of(const RowArgs& a, int b) {
 }
 __device__ __forceinline__ int ld_acquire(const int* p) {
     int v; asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
+}
+// The draw of a sequence is decided: count it (high half), and when it goes to the fp64 re-draw take its place in
+// the list (low half).  One word, so that a reader who sees all sequences decided also sees the final list length.
+__device__ __forceinline__ void draw_decided(unsigned long long* w) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(w), "l"(1ull << 32) : "memory");
+}
+__device__ __forceinline__ int draw_listed(unsigned long long* w) {
+    return (int)(atomicAdd(w, (1ull << 32) | 1ull) & 0xffffffffull);
 }
 // Workspace records written by other CTAs of this launch are read through L2 only: the L1 of this SM
 // may hold an older copy of the line (a neighbouring record read earlier).

@@ -7,24 +7,32 @@ namespace bebop {
 namespace {
 
 // ------------------------------------------------------------------ fp64 re-draw of the listed sequences
-// Two small kernels behind the pipelined kernel, for the few sequences whose fast draw did not clear its
+// One small kernel beside the pipelined kernel, for the few sequences whose fast draw did not clear its
 // error bound.  Every row is cut into XT = 4T quarter slices; the work items (listed sequence, quarter
-// slice) are dealt round-robin to a fixed grid.  Everything is evaluated in double around the row
-// exponents that phase A left (any common reference cancels in p = a / sum a).
-//   k_redraw_sum   exact normalisers: sum of exponentials of each quarter slice of the draw rows;
-//   k_redraw_mass  residual mass of each quarter slice, one sum per warp (warp w owns the contiguous
-//                  vectors [w*cw, (w+1)*cw)); the CTA that completes a sequence picks its token at
-//                  once: quarter slice and warp chunk from the stored sums, then the few hundred
-//                  tokens of that chunk are evaluated once more, one or two per thread, and scanned.
+// slice) are dealt round-robin to a grid that fits the device at once.  Everything is evaluated in double
+// around the row exponents that phase A left (any common reference cancels in p = a / sum a).  An item is
+//   sum    exact normalisers: sum of exponentials of its quarter slice of the draw rows; then, once
+//          the sums of all quarter slices of the sequence are there (a counter per listed sequence),
+//   mass   residual mass of the quarter slice, one sum per warp (warp w owns the contiguous vectors
+//          [w*cw, (w+1)*cw)); the CTA that completes a sequence picks its token at once: quarter slice
+//          and warp chunk from the stored sums, then the few hundred tokens of that chunk are evaluated
+//          once more, one or two per thread, and scanned.
+// The kernel is a programmatic dependent of the pipelined kernel that does NOT wait for that grid: its
+// CTAs move in as CTAs of the main kernel leave, and work through the list while it still grows (records
+// carry a mark; one word counts the listed sequences and the sequences whose draw is decided, which tells the
+// end of the list).  The sequences
+// listed early are finished before the main kernel ends.
 struct RedrawArgs {
     RowArgs r;
     const float* u_final;
     VerifyOut o;
-    const int* fb_count;     // listed sequences
-    const FbRec* fb_list;
-    const int* wait_failed;  // set by a device-side wait of the main kernel that gave up
+    const unsigned long long* fb_count;   // low half: listed sequences so far; high half: sequences whose draw is decided
+    const FbRec* fb_list;    // records, valid once their b1 is non-zero
+    int expect;              // sequences that get decided: the list is complete when the high half reaches it
+    int* wait_failed;        // set by a device-side wait that gave up
     double2* xsum;           // [B][XT] sums of exponentials (target row, draft row) per quarter slice
     double* xmass;           // [B][XT][WW] residual mass per quarter slice and warp chunk
+    int* xsdone;             // [B] per listed sequence: sum tasks finished
     int* xdone;              // [B] per listed sequence: mass tasks finished
     int T, slice_vecs;
 };
@@ -33,6 +41,9 @@ struct RedrawArgs {
 // 2^f by its series to the fifth power (the next term is below 4e-17 of the result).  About a dozen
 // double-precision instructions, a third of the library routine; the result is within 2 ulp.
 // `tab` holds 2^(j/64), j = 0..63, in shared memory.  Arguments below -1000 (and -inf) give 0.
+#ifndef BEBOP_XPOLL
+#define BEBOP_XPOLL 256
+#endif
 constexpr int XTAB = 64;
 __device__ __forceinline__ void x_exp2_table(double* tab) {
     if (threadIdx.x < XTAB) tab[threadIdx.x] = exp2((double)threadIdx.x * (1.0 / XTAB));
@@ -68,8 +79,8 @@ __device__ __forceinline__ double x_resid(const XRow& d, float zp, float zq, con
 }
 __device__ __forceinline__ void x_row(const RedrawArgs& a, int slot, XRow* d) {
     const RowArgs& R = a.r;
-    const FbRec rec = a.fb_list[slot];
-    const int b = rec.b, k = rec.kp >> 1;
+    const FbRec rec = ld_cg(a.fb_list + slot);
+    const int b = rec.b1 - 1, k = rec.kp >> 1;
     d->b = b; d->k = k;
     d->pair = rec.kp & 1;
     d->prow = row_ptr(R, b, k);
@@ -79,8 +90,8 @@ __device__ __forceinline__ void x_row(const RedrawArgs& a, int slot, XRow* d) {
     d->eq = (double)rec.eq;
     d->ip = 1.0; d->iq = 1.0;
 }
-constexpr int kRedrawGrid = 148 * 4;
-constexpr int XNU = 2;     // vectors per thread and row in a quarter slice (at most 512 vectors)
+constexpr int XNU = (kPipeSliceVecs / kRedrawCut + WT - 1) / WT;     // vectors per thread and row in a work item
+static_assert(kPipeSliceVecs % (kRedrawCut * 2) == 0 && XNU >= 1 && XNU <= 2, "work items of the fp64 re-draw");
 
 // this thread's vectors of quarter slice s: warp chunk [warp*cw, warp*cw + cw), lanes interleaved
 template <int DT>
@@ -88,7 +99,7 @@ __device__ __forceinline__ void x_load(const RedrawArgs& a, const XRow& d, int s
                                        float (*fq)[Elem<DT>::VEC]) {
     constexpr int VEC = Elem<DT>::VEC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int qv = a.slice_vecs >> 2, cw = (qv + WW - 1) / WW;
+    const int qv = a.slice_vecs / kRedrawCut, cw = (qv + WW - 1) / WW;
     const int v0 = s * qv, nv = max(min(qv, a.r.nvec - v0), 0);
 #pragma unroll
     for (int u = 0; u < XNU; ++u) {
@@ -103,52 +114,8 @@ __device__ __forceinline__ void x_load(const RedrawArgs& a, const XRow& d, int s
     }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(WT) k_redraw_sum(const RedrawArgs a) {
-    constexpr int VEC = Elem<DT>::VEC;
-    __shared__ double sh[2][WW];
-    __shared__ double tab[XTAB];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // launched as a programmatic dependent of the main kernel: set up, then wait for that grid's completion
-    x_exp2_table(tab);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int XT = 4 * a.T, items = *a.fb_count * XT;
-    // a wait of the main kernel that gave up: every row's status says so
-    if (a.o.row_status && *a.wait_failed) {
-        for (int b = blockIdx.x * WT + tid; b < a.r.B; b += gridDim.x * WT) a.o.row_status[b] |= ST_WAIT;
-    }
-    if ((int)blockIdx.x >= items) return;
-    __syncthreads();
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        const int slot = item / XT, s = item - slot * XT;
-        XRow d;
-        x_row(a, slot, &d);
-        float fp[XNU][VEC], fq[XNU][VEC];
-        x_load<DT>(a, d, s, fp, fq);
-        double sa = 0.0, sb = 0.0;
-#pragma unroll
-        for (int u = 0; u < XNU; ++u) {
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                sa += x_exp2(fma((double)fp[u][i], d.c, -d.ep), tab);
-                if (d.pair) sb += x_exp2(fma((double)fq[u][i], d.c, -d.eq), tab);
-            }
-        }
-        sa = warp_sum(sa); sb = warp_sum(sb);
-        __syncthreads();
-        if (lane == 0) { sh[0][warp] = sa; sh[1][warp] = sb; }
-        __syncthreads();
-        if (tid == 0) {
-            double ta = 0.0, tb = 0.0;
-            for (int w = 0; w < WW; ++w) { ta += sh[0][w]; tb += sh[1][w]; }
-            a.xsum[(int64_t)d.b * XT + s] = make_double2(ta, tb);
-        }
-    }
-}
-
 struct PickShared {
-    double part[4 * MAX_SLICES];     // slice masses of the sequence, later the warp masses of one slice
+    double part[kRedrawCut * MAX_SLICES];     // slice masses of the sequence, later the warp masses of one slice
     double redd[WW];
     double base, target;
     int last, sel, chunk, tok_first, tok_last;
@@ -173,38 +140,111 @@ __device__ __forceinline__ int pick_entry(const double* m, int n, double t, doub
     return last;
 }
 
+__device__ __forceinline__ unsigned long long x_ld_count(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+// 1: slot is listed and its record is valid; 0: the list is complete and ends before it; -1: a wait gave up
+__device__ __forceinline__ int x_wait_slot(const RedrawArgs& a, int slot) {
+    uint32_t i = 0;
+    for (; i < kSpin; ++i) {
+        const unsigned long long w = x_ld_count(a.fb_count);
+        if (slot < (int)(w & 0xffffffffull)) break;
+        if ((int)(w >> 32) >= a.expect) return 0;
+        __nanosleep(BEBOP_XPOLL);
+    }
+    if (i == kSpin) return -1;
+    for (i = 0; i < kSpin; ++i) {                       // a place in the list is taken before its record is written
+        if (ld_cg(a.fb_list + slot).b1 != 0) return 1;
+        __nanosleep(64);
+    }
+    return -1;
+}
+
 template <int DT>
-__global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
+__global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
     constexpr int VEC = Elem<DT>::VEC;
     __shared__ PickShared S;
+    __shared__ double sh[2][WW];
     __shared__ double tab[XTAB];
+    __shared__ int go;
+    extern __shared__ double xe[];       // [2][XNU * VEC][WT] exponentials of this item's elements (target row, draft row)
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     x_exp2_table(tab);
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // programmatic dependent of k_redraw_sum
-    const int K = R.K, XT = 4 * a.T, items = *a.fb_count * XT;
-    const int qv = a.slice_vecs >> 2, cw = (qv + WW - 1) / WW;
-    if ((int)blockIdx.x >= items) return;
+    const int K = R.K, XT = kRedrawCut * a.T;
+    const int qv = a.slice_vecs / kRedrawCut, cw = (qv + WW - 1) / WW;
+    const long items_max = (long)R.B * XT;
     __syncthreads();
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        const int slot = item / XT, s = item - slot * XT;
+    for (long item = blockIdx.x; item < items_max; item += gridDim.x) {
+        const int slot = (int)(item / XT), s = (int)(item - (long)slot * XT);
+        if (tid == 0) go = x_wait_slot(a, slot);
+        __syncthreads();
+        const int g = go;
+        __syncthreads();
+        if (g <= 0) {                                   // slots come in rising order: nothing behind this one either
+            if (g < 0 && tid == 0) atomicExch(a.wait_failed, 1);
+            break;
+        }
         XRow d;
         x_row(a, slot, &d);
         const int b = d.b;
-        // exact normalisers: every warp adds the quarter-slice sums in the same order (lane t takes sums t,
-        // t + 32, ...; the butterfly leaves the same bits in every lane), so every CTA gets the same value
-        double Sa = 0.0, Sb = 0.0;
-        for (int t = lane; t < XT; t += 32) { const double2 x = a.xsum[(int64_t)b * XT + t]; Sa += x.x; Sb += x.y; }
-        Sa = warp_sum(Sa); Sb = warp_sum(Sb);
-        d.ip = 1.0 / Sa; d.iq = d.pair ? 1.0 / Sb : 0.0;
-        if (d.pair) {     // a bonus row needs no mass pass: its masses are sums of exponentials over Sa
+        // ---- sum of exponentials of this quarter slice
+        {
             float fp[XNU][VEC], fq[XNU][VEC];
             x_load<DT>(a, d, s, fp, fq);
-            double m = 0.0;
+            double sa = 0.0, sb = 0.0;
 #pragma unroll
             for (int u = 0; u < XNU; ++u) {
 #pragma unroll
-                for (int i = 0; i < VEC; ++i) m += x_resid(d, fp[u][i], fq[u][i], tab);
+                for (int i = 0; i < VEC; ++i) {
+                    const double ea = x_exp2(fma((double)fp[u][i], d.c, -d.ep), tab);
+                    sa += ea;
+                    if (d.pair) {
+                        const double eb = x_exp2(fma((double)fq[u][i], d.c, -d.eq), tab);
+                        sb += eb;
+                        // kept for the mass pass, which then needs neither the rows nor the exponentials again
+                        xe[(u * VEC + i) * WT + tid] = ea;
+                        xe[((XNU + u) * VEC + i) * WT + tid] = eb;
+                    }
+                }
+            }
+            sa = warp_sum(sa); sb = warp_sum(sb);
+            if (lane == 0) { sh[0][warp] = sa; sh[1][warp] = sb; }
+            __syncthreads();
+            if (tid == 0) {
+                double ta = 0.0, tb = 0.0;
+                for (int w = 0; w < WW; ++w) { ta += sh[0][w]; tb += sh[1][w]; }
+                a.xsum[(int64_t)b * XT + s] = make_double2(ta, tb);
+                __threadfence();
+                atomicAdd(a.xsdone + slot, 1);
+                // ... and wait (bounded) for the other quarter slices of the sequence
+                go = spin_ge(a.xsdone + slot, XT) ? 1 : 0;
+            }
+            __syncthreads();
+            const int ok = go;
+            __syncthreads();
+            if (!ok) {
+                if (tid == 0) { atomicExch(a.wait_failed, 1); if (a.o.row_status) atomicOr(a.o.row_status + b, ST_WAIT); }
+                continue;
+            }
+        }
+        // exact normalisers: every warp adds the quarter-slice sums in the same order (lane t takes sums t,
+        // t + 32, ...; the butterfly leaves the same bits in every lane), so every CTA gets the same value
+        double Sa = 0.0, Sb = 0.0;
+        for (int t = lane; t < XT; t += 32) { const double2 x = __ldcg(a.xsum + (int64_t)b * XT + t); Sa += x.x; Sb += x.y; }
+        Sa = warp_sum(Sa); Sb = warp_sum(Sb);
+        d.ip = 1.0 / Sa; d.iq = d.pair ? 1.0 / Sb : 0.0;
+        if (d.pair) {     // a bonus row needs no mass pass: its masses are sums of exponentials over Sa
+            double m = 0.0;
+#pragma unroll
+            for (int j = 0; j < XNU * VEC; ++j) {
+                // as x_resid, from the stored exponentials (explicit roundings: see there)
+                const double p = __dmul_rn(xe[j * WT + tid], d.ip);
+                const double q = __dmul_rn(xe[(XNU * VEC + j) * WT + tid], d.iq);
+                const double df = p - q;
+                m += df > 0.0 ? df : 0.0;
             }
             m = warp_sum(m);
             if (lane == 0) a.xmass[((int64_t)b * XT + s) * WW + warp] = m;
@@ -224,7 +264,7 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
             for (int t = tid; t < XT; t += WT) {
                 double m = 0.0;
                 if (d.pair) { for (int w = 0; w < WW; ++w) m += __ldcg(a.xmass + ((int64_t)b * XT + t) * WW + w); }
-                else m = a.xsum[(int64_t)b * XT + t].x * d.ip;
+                else m = __ldcg(a.xsum + (int64_t)b * XT + t).x * d.ip;
                 S.part[t] = m;
             }
             __syncthreads();
@@ -240,7 +280,12 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
             __syncthreads();
         }
         if (tid == 0) {
-            if (zero_resid && a.o.row_status) a.o.row_status[b] |= ST_ZERO_RESID;
+            if (zero_resid && a.o.row_status) {
+                // the main kernel writes this row's status word once, with a plain store: add the bit only when
+                // that grid is through (rare, and then a wait of some microseconds at most)
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                atomicOr(a.o.row_status + b, ST_ZERO_RESID);
+            }
             const double t = (double)a.u_final[b] * S.base;
             double C = 0.0;
             S.sel = pick_entry(S.part, XT, t, &C);
@@ -316,6 +361,12 @@ __global__ void __launch_bounds__(WT) k_redraw_mass(const RedrawArgs a) {
         if (tid == 0) a.o.out_tokens[(int64_t)b * (K + 1) + d.k] = S.tok_first != 0x7fffffff ? S.tok_first : S.tok_last;
         __syncthreads();
     }
+    // a wait that gave up, in the main kernel or here: every row's status says so
+    if (a.o.row_status) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // the main grid is through and its writes are visible
+        if (ld_acquire(a.wait_failed) != 0)
+            for (int b = blockIdx.x * WT + tid; b < R.B; b += gridDim.x * WT) atomicOr(a.o.row_status + b, ST_WAIT);
+    }
 }
 
 }  // namespace
@@ -325,32 +376,58 @@ void wave_set_trace(long long* p) { g_wave_trace = p; }
 cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 void wave_set_events(cudaEvent_t start, cudaEvent_t stop) { g_ev_start = start; g_ev_stop = stop; }
 
-// fp64 re-draw of the listed sequences (usually a few per cent of the batch; the count stays on the device)
-cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const int* fb_count,
-                          const FbRec* fb_list, const int* wait_failed, char* w, const WavePlan& wp,
-                          cudaStream_t stream) {
+namespace {
+template <int DT>
+constexpr size_t redraw_smem() { return sizeof(double) * 2 * XNU * Elem<DT>::VEC * WT; }
+template <int DT>
+int redraw_grid() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
+    int per_sm = 0, sms = 0;
+    if (cudaFuncSetAttribute(k_redraw<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)redraw_smem<DT>()) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_redraw<DT>, WT, redraw_smem<DT>()) != cudaSuccess) per_sm = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaGetLastError();
+    const int n = per_sm * sms;
+    if (dev >= 0 && dev < 64) cached[dev] = n;
+    return n;
+}
+}  // namespace
+
+// fp64 re-draw of the listed sequences (usually a few per cent of the batch; the count stays on the device).
+// `expect` sequences get their draw decided by the main kernel (0: none, nothing is listed).
+cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const unsigned long long* fb_count,
+                          const FbRec* fb_list, int expect, int* wait_failed, char* w,
+                          const WavePlan& wp, cudaStream_t stream) {
     RedrawArgs ra;
     ra.r = a; ra.u_final = u_final; ra.o = o;
-    ra.fb_count = fb_count; ra.fb_list = fb_list; ra.wait_failed = wait_failed;
+    ra.fb_count = fb_count; ra.fb_list = fb_list; ra.expect = expect;
+    ra.wait_failed = wait_failed;
     ra.xsum = reinterpret_cast<double2*>(w + wp.off_xsum);
     ra.xmass = reinterpret_cast<double*>(w + wp.off_xmass);
+    ra.xsdone = reinterpret_cast<int*>(w + wp.off_xsdone);
     ra.xdone = reinterpret_cast<int*>(w + wp.off_xdone);
     ra.T = wp.T; ra.slice_vecs = wp.slice_vecs;
-    // the count of listed sequences stays on the device: a fixed grid, four CTAs per SM, takes the work
-    // items round-robin (a CTA without an item returns at once)
-    const long items_max = (long)a.B * 4 * wp.T;
-    const int grid = (int)(items_max < kRedrawGrid ? items_max : kRedrawGrid);
-    // each kernel may be scheduled while its predecessor in the stream drains; it waits inside for that
-    // grid's completion (griddepcontrol.wait) before it reads what the predecessor wrote
+    // CTAs of this grid wait for one another (the sums of a sequence come from many of them): the grid
+    // must fit the device at once.  A CTA takes the work items round-robin.
+    const int cap = a.dt == 0 ? redraw_grid<0>() : redraw_grid<1>();
+    if (cap < 1) return cudaErrorLaunchOutOfResources;
+    const long items_max = (long)a.B * kRedrawCut * wp.T;
+    const int grid = (int)(items_max < cap ? items_max : cap);
+    // scheduled as soon as the main kernel lets go of SMs; it does not wait for that grid as a whole
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(WT); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(WT); cfg.stream = stream;
+    cfg.dynamicSmemBytes = a.dt == 0 ? redraw_smem<0>() : redraw_smem<1>();
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = a.dt == 0 ? cudaLaunchKernelEx(&cfg, k_redraw_sum<0>, ra) : cudaLaunchKernelEx(&cfg, k_redraw_sum<1>, ra);
-    if (e != cudaSuccess) return e;
-    return a.dt == 0 ? cudaLaunchKernelEx(&cfg, k_redraw_mass<0>, ra) : cudaLaunchKernelEx(&cfg, k_redraw_mass<1>, ra);
+    return a.dt == 0 ? cudaLaunchKernelEx(&cfg, k_redraw<0>, ra) : cudaLaunchKernelEx(&cfg, k_redraw<1>, ra);
 }
 
 }  // namespace bebop
