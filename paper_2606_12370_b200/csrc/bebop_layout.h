@@ -21,6 +21,7 @@ struct alignas(16) FbRec {
 #define BEBOP_REDRAW_CUT 4
 #endif
 constexpr int kRedrawCut = BEBOP_REDRAW_CUT;   // the fp64 re-draw cuts every row slice into so many work items
+constexpr size_t kRedrawTicketOffset = 192;   // unsigned: next work item of the fp64 re-draw (zeroed head of the workspace)
 constexpr size_t kFbCountOffset = 128;   // 8 bytes inside the zeroed head of the workspace: low int, sequences listed for the fp64
                                          // re-draw; high int, sequences whose draw is decided
 struct WavePlan {

@@ -9,7 +9,7 @@ namespace {
 // ------------------------------------------------------------------ fp64 re-draw of the listed sequences
 // One small kernel beside the pipelined kernel, for the few sequences whose fast draw did not clear its
 // error bound.  Every row is cut into XT = 4T quarter slices; the work items (listed sequence, quarter
-// slice) are dealt round-robin to a grid that fits the device at once.  Everything is evaluated in double
+// slice) are taken from a counter by a grid that fits the device at once.  Everything is evaluated in double
 // around the row exponents that phase A left (any common reference cancels in p = a / sum a).  An item is
 //   sum    exact normalisers: sum of exponentials of its quarter slice of the draw rows; then, once
 //          the sums of all quarter slices of the sequence are there (a counter per listed sequence),
@@ -34,6 +34,7 @@ struct RedrawArgs {
     double* xmass;           // [B][XT][WW] residual mass per quarter slice and warp chunk
     int* xsdone;             // [B] per listed sequence: sum tasks finished
     int* xdone;              // [B] per listed sequence: mass tasks finished
+    unsigned* xticket;       // [1] next work item
     int T, slice_vecs;
 };
 
@@ -169,6 +170,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
     __shared__ double sh[2][WW];
     __shared__ double tab[XTAB];
     __shared__ int go;
+    __shared__ unsigned item_sh;
     extern __shared__ double xe[];       // [2][XNU * VEC][WT] exponentials of this item's elements (target row, draft row)
     const RowArgs& R = a.r;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -177,11 +179,18 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
     const int qv = a.slice_vecs / kRedrawCut, cw = (qv + WW - 1) / WW;
     const long items_max = (long)R.B * XT;
     __syncthreads();
-    for (long item = blockIdx.x; item < items_max; item += gridDim.x) {
-        const int slot = (int)(item / XT), s = (int)(item - (long)slot * XT);
-        if (tid == 0) go = x_wait_slot(a, slot);
+    // Work items are taken in order from a ticket counter, so the CTAs that are on the device work on the oldest
+    // listed sequence; whoever holds an item is running, so the wait for a sequence's other items cannot
+    // depend on a CTA that has not started.
+    for (;;) {
+        if (tid == 0) {
+            const unsigned item = atomicAdd(a.xticket, 1u);
+            item_sh = item;
+            go = item < (unsigned long)items_max ? x_wait_slot(a, (int)(item / (unsigned)XT)) : 0;
+        }
         __syncthreads();
         const int g = go;
+        const int slot = (int)(item_sh / (unsigned)XT), s = (int)(item_sh - (unsigned)slot * (unsigned)XT);
         __syncthreads();
         if (g <= 0) {                                   // slots come in rising order: nothing behind this one either
             if (g < 0 && tid == 0) atomicExch(a.wait_failed, 1);
@@ -412,9 +421,10 @@ cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, c
     ra.xmass = reinterpret_cast<double*>(w + wp.off_xmass);
     ra.xsdone = reinterpret_cast<int*>(w + wp.off_xsdone);
     ra.xdone = reinterpret_cast<int*>(w + wp.off_xdone);
+    ra.xticket = reinterpret_cast<unsigned*>(w + kRedrawTicketOffset);
     ra.T = wp.T; ra.slice_vecs = wp.slice_vecs;
-    // CTAs of this grid wait for one another (the sums of a sequence come from many of them): the grid
-    // must fit the device at once.  A CTA takes the work items round-robin.
+    // CTAs of this grid wait for one another (the sums of a sequence come from kRedrawCut * T of them), so
+    // the grid is at most what fits the device at once; a CTA takes work items from a counter.
     const int cap = a.dt == 0 ? redraw_grid<0>() : redraw_grid<1>();
     if (cap < 1) return cudaErrorLaunchOutOfResources;
     const long items_max = (long)a.B * kRedrawCut * wp.T;
