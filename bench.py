@@ -245,7 +245,7 @@ def run_ours(args):
     kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
     kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = 6 if args.path == 1 else 3      # main kernel, 2 fp64 re-draw kernels | 6 general kernels
+    launches_per_call = 6 if args.path == 1 else 2      # main kernel, fp64 re-draw kernel | 6 general kernels
 
     # the same call without a TV output (the second sweep then reads only the rows a token is drawn from): not the
     # headline, which emits TV; reported beside it

@@ -4,6 +4,25 @@
 
 namespace bebop {
 
+#ifdef BEBOP_TRACE
+// timeline of the re-draw kernel: [2i] earliest, [2i+1] latest global-timer stamp of event i over all CTAs
+__device__ unsigned long long g_redraw_trace[32];
+__device__ __forceinline__ void xt_log(int i) {
+    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(&g_redraw_trace[2 * i], t); atomicMax(&g_redraw_trace[2 * i + 1], t);
+}
+#define XTLOG(i) do { if (threadIdx.x == 0) xt_log(i); } while (0)
+extern "C" void bebop_debug_redraw_trace(unsigned long long* host32, int reset) {
+    if (reset) {
+        unsigned long long init[32];
+        for (int i = 0; i < 16; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
+        cudaMemcpyToSymbol(g_redraw_trace, init, sizeof(init));
+    } else cudaMemcpyFromSymbol(host32, g_redraw_trace, 32 * sizeof(unsigned long long));
+}
+#else
+#define XTLOG(i) do { } while (0)
+#endif
+
 namespace {
 
 // ------------------------------------------------------------------ fp64 re-draw of the listed sequences
@@ -196,6 +215,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             if (g < 0 && tid == 0) atomicExch(a.wait_failed, 1);
             break;
         }
+        XTLOG(0);
         XRow d;
         x_row(a, slot, &d);
         const int b = d.b;
@@ -222,6 +242,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             sa = warp_sum(sa); sb = warp_sum(sb);
             if (lane == 0) { sh[0][warp] = sa; sh[1][warp] = sb; }
             __syncthreads();
+            XTLOG(1);
             if (tid == 0) {
                 double ta = 0.0, tb = 0.0;
                 for (int w = 0; w < WW; ++w) { ta += sh[0][w]; tb += sh[1][w]; }
@@ -241,6 +262,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
         }
         // exact normalisers: every warp adds the quarter-slice sums in the same order (lane t takes sums t,
         // t + 32, ...; the butterfly leaves the same bits in every lane), so every CTA gets the same value
+        XTLOG(3);
         double Sa = 0.0, Sb = 0.0;
         for (int t = lane; t < XT; t += 32) { const double2 x = __ldcg(a.xsum + (int64_t)b * XT + t); Sa += x.x; Sb += x.y; }
         Sa = warp_sum(Sa); Sb = warp_sum(Sb);
@@ -264,6 +286,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             S.last = atomicAdd(a.xdone + slot, 1) == XT - 1;
         }
         __syncthreads();
+        XTLOG(4);
         if (!S.last) continue;
         __threadfence();
 
@@ -301,6 +324,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             S.target = t; S.base = C;
         }
         __syncthreads();
+        XTLOG(5);
         const int qs = S.sel;
         // Stage 2: warp chunk inside the quarter slice (residual: stored; plain softmax row: evaluated now)
         const int p0 = qs * qv, pn = max(min(qv, R.nvec - p0), 0);
@@ -368,6 +392,7 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
         if (lastpos >= 0) atomicMax(&S.tok_last, lastpos);
         __syncthreads();
         if (tid == 0) a.o.out_tokens[(int64_t)b * (K + 1) + d.k] = S.tok_first != 0x7fffffff ? S.tok_first : S.tok_last;
+        XTLOG(7);
         __syncthreads();
     }
     // a wait that gave up, in the main kernel or here: every row's status says so
