@@ -109,6 +109,31 @@ def test_many_short_sequences_finish_in_quick_succession():
     full_check(cfg, sample=256)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_every_sequence_goes_to_the_fp64_redraw(dtype, kernel_path):
+    """A target u * Z next to zero sits inside the error bound of the fp32 prefix sum, so no fast draw is kept:
+    every sequence is listed while the pipelined kernel still runs, and the re-draw kernel has more work items
+    than CTAs.  The token is the first one with residual mass (bonus rows: with probability), exactly."""
+    cfg = G.Config("redraw_all", 600, 2, 20000, dtype, 2.0, True, 1.0, 1.0, seed=41)
+    x = G.make_inputs(cfg, DEV)
+    x["draft_len"] = torch.tensor([i % 3 for i in range(cfg.B)], dtype=torch.int32, device=DEV)
+    x["u_final"] = torch.full((cfg.B,), 1e-30, dtype=torch.float32, device=DEV)
+    got = run_verify(x)
+    got = run_verify(x, workspace=got["workspace"])     # the second call finds the first call's records there
+    torch.cuda.synchronize()
+    if kernel_path == "pipe":
+        off = P.bebop_debug_fallback_offset(cfg.B, cfg.K, cfg.V, 0 if dtype == "f32" else 1)
+        assert int(got["workspace"][off:off + 4].view(torch.int32).item()) == cfg.B
+    check_properties(got, x)
+    idx = np.unique(np.linspace(0, cfg.B - 1, 96).astype(np.int64))
+    ref = oracle_on(x, idx)
+    # (the oracle flags every one of these draws as a near-tie of the inverse CDF, which it is; the first token
+    # with mass is unique all the same, so the comparison is exact here)
+    assert np.array_equal(to_np(got["accept_len"])[idx], ref["accept_len"])
+    assert np.array_equal(to_np(got["out_tokens"])[idx], ref["out_tokens"])
+    assert np.abs(to_np(got["tv"])[idx] - ref["tv"]).max() <= TOL[dtype]
+
+
 def test_all_draft_lengths_including_zero():
     cfg = G.Config("len", 10, 4, 4096, "f32", 2.0, False, 0.3, 1.0, seed=5)
     x = G.make_inputs(cfg, DEV)
