@@ -26,7 +26,7 @@ constexpr size_t kFbCountOffset = 128;   // 8 bytes inside the zeroed head of th
                                          // re-draw; high int, sequences whose draw is decided
 struct WavePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 16)
-    size_t off_p1done, off_p2done, off_xdone, off_xsdone, off_fbrec, off_rowcnt, zero_bytes;
+    size_t off_p1done, off_p2done, off_ddone, off_xdone, off_xsdone, off_fbrec, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
     size_t off_part, off_rstat, off_dpart, off_tvacc, off_sacc, off_sinfo, total;
 };
@@ -59,6 +59,7 @@ static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_
     size_t o = 256;                                           // ticket, wait flag; at kFbCountOffset the re-draw count
     w.off_p1done = o; o += align256(sizeof(int) * (size_t)B);      // per sequence: rows merged
     w.off_p2done = o; o += align256(sizeof(int) * (size_t)B);
+    w.off_ddone = o;  o += align256(sizeof(int) * (size_t)B);      // per sequence: partials of the draw row
     w.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
     w.off_xsdone = o; o += align256(sizeof(int) * (size_t)B);
     w.off_fbrec = o;  o += align256(16 * (size_t)B);          // records of the sequences whose draw goes to fp64

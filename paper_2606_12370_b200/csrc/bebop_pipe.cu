@@ -69,10 +69,6 @@ constexpr int STAGE_BYTES = PSLICE * 16;
 #ifndef BEBOP_PIPE_NOHINT
 #define BEBOP_PIPE_NOHINT 0
 #endif
-#ifndef BEBOP_PIPE_LAG_MB
-#define BEBOP_PIPE_LAG_MB 0
-#endif
-constexpr size_t kLagBytes = (size_t)BEBOP_PIPE_LAG_MB << 20;   // logits between the first sweep and the second
 constexpr int kPend = 4;                          // runs a producer may set aside
 #ifndef BEBOP_PIPE_BATCH
 #define BEBOP_PIPE_BATCH 5
@@ -203,35 +199,42 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     // (a caller that asks for no TV needs the second sweep over one row per sequence only: the one a token is drawn from)
     // (and bebop_tv has the K row pairs and no bonus row)
     // (the greedy mode sweeps the K + 1 target rows once)
-    const int c0 = (GRD ? K + 1 : NR) * T, c2 = GRD ? 0 : (TVO ? K : (a.o.tv ? K + 1 : 1)) * T2;
-    const double inv_c0 = 1.0 / c0, inv_c2 = GRD ? 0.0 : 1.0 / c2, inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
+    // The second sweep comes in two passes: first the row each sequence's token is drawn from (so that every draw,
+    // and the list of the sequences that go to the fp64 re-draw, is done early in the sweep), then the other
+    // rows, which only TV needs.  bebop_tv has the K row pairs and no draw; the greedy mode sweeps the K + 1 target
+    // rows once.
+    const int c0 = (GRD ? K + 1 : NR) * T;
+    const int c2a = (GRD || TVO) ? 0 : T2, c2b = GRD ? 0 : ((TVO || a.o.tv) ? K * T2 : 0);
+    const double inv_c0 = 1.0 / c0, inv_c2a = c2a ? 1.0 / c2a : 0.0, inv_c2b = c2b ? 1.0 / c2b : 0.0;
+    const double inv_T = 1.0 / T, inv_T2 = 1.0 / T2;
     const int sv1 = a.slice_vecs, sv2 = a.slice_vecs >> 1;
-    // Ticket order: block i = 0, 1, .. holds P1 of sequence i, then P2 of sequence i - W (each where the sequence
-    // exists).  With W = B (the default) that is all of P1, then all of P2: two full sweeps, sequences ascending,
-    // so that the first sequences' accept scans are long done when the second sweep starts.  A smaller W pairs
-    // the sweeps (the second finds some of its logits still in L2: the first sweep asks L2 to keep them, the
-    // second to drop them) at the price of waiting.
-    const int W = a.lag;
+    // Ticket order: blocks 0 .. B-1 hold the first sweep of sequence i, blocks B .. 2B-1 the first pass of the
+    // second sweep, blocks 2B .. 3B-1 its second pass: full sweeps, sequences ascending, so that a sequence's
+    // accept scan is long done when the second sweep reaches it.  (Pairing the sweeps so that the second finds
+    // its logits in L2 was measured and dropped: it waited for accept scans more than the L2 hits saved.)
     const unsigned long long pol_keep = l2_policy(true), pol_drop = l2_policy(false);
     auto clampB = [&](int x) { return x < 0 ? 0 : (x > B ? B : x); };
-    auto before = [&](int i) { return c0 * clampB(i) + c2 * clampB(i - W); };   // tickets before block i
+    auto before = [&](int i) { return c0 * clampB(i) + c2a * clampB(i - B) + c2b * clampB(i - 2 * B); };   // tickets before block i
     int blk = 0, f_here = 0, f_next = before(1);      // tickets of this CTA only grow: the block is tracked, not searched
     // the run of consecutive tasks of one sequence and phase that starts at ticket t, at most `want` tasks;
-    // Run.wv is the sequence, Run.off the offset inside the sequence's block of that phase
+    // Run.wv is the sequence, Run.off the offset inside the sequence's tasks of that phase (second sweep: the draw row
+    // is row 0, the other rows follow)
+    const int t1 = B * c0, t2 = t1 + B * c2a;
     auto decode = [&](int t, int want) {
-        if (W >= B && f_next <= t) {
-            // two full sweeps: the block follows from one division (a CTA's next tickets are some thirty blocks
-            // on: stepping there one block at a time was most of what the producer did between two runs)
-            blk = (GRD || t < B * c0) ? div_by(t, c0, inv_c0) : B + div_by(t - B * c0, c2, inv_c2);
+        if (f_next <= t) {
+            // the block follows from one division (a CTA's next tickets are some thirty blocks on: stepping there
+            // one block at a time was most of what the producer did between two runs)
+            blk = (GRD || t < t1) ? div_by(t, c0, inv_c0)
+                                  : (t < t2 ? B + div_by(t - t1, c2a, inv_c2a) : 2 * B + div_by(t - t2, c2b, inv_c2b));
             f_here = before(blk); f_next = before(blk + 1);
         }
         while (f_next <= t) { ++blk; f_here = f_next; f_next = before(blk + 1); }
         Run r;
-        int o = t - f_here, room;
-        const int n0 = blk < B ? c0 : 0;
-        if (o < n0) { r.ph = 0; r.wv = blk; r.off = o; room = n0 - o; }
-        else { r.ph = 2; r.wv = blk - W; r.off = o - n0; room = n0 + c2 - o; }
-        r.cnt = min(want, room);
+        const int o = t - f_here;
+        if (blk < B) { r.ph = 0; r.wv = blk; r.off = o; }
+        else if (blk < 2 * B) { r.ph = 2; r.wv = blk - B; r.off = o; }
+        else { r.ph = 2; r.wv = blk - 2 * B; r.off = o + c2a; }
+        r.cnt = min(want, f_next - t);
         return r;
     };
     // Is sequence b ready for the phase?  P2 needs its accept scan.  A run that is not ready is set aside (up to
@@ -353,7 +356,10 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
             } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
                 const SeqInfo si = seen_b == b ? seen : ld_cg(a.sinfo + b);
-                const int k = a.o.tv ? r : max(si.draw_row, 0);
+                // row 0 of the sequence's second sweep is the row its token is drawn from; the others follow in order
+                const bool drawrow = !TVO && r == 0;
+                const int rp = TVO ? r : r - 1;
+                const int k = drawrow ? max(si.draw_row, 0) : (TVO ? rp : rp + (rp >= si.draw_row ? 1 : 0));
                 d.r = k;
                 RowStat sp = ld_cg(a.rstat + (int64_t)b * NR + k);
                 RowStat sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + min(k, K - 1));
@@ -365,12 +371,12 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
                 d.c = __int_as_float(si.pad0);
                 const bool pair = k < L;
-                skip = k > L || si.n < 0 || (!pair && si.draw_row != L) || no_row_k;
+                skip = k > L || si.n < 0 || (!pair && !(drawrow && si.draw_row == L)) || no_row_k;
                 // the sequence's second sweep: every half slice of the L row pairs, and of the bonus row if drawn from
                 d.need = T2 * (L + (si.draw_row == L ? 1 : 0));
                 if (!a.o.tv) d.need = T2;
                 if (!skip) {
-                    d.flags = (pair ? 1 : 0) | (si.draw_row == k ? 2 : 0);
+                    d.flags = (pair ? 1 : 0) | (drawrow ? 2 : 0);
                     d.P = row_scale(sp);
                     if (pair) d.Q = row_scale(sq);
                     row0 = row_ptr(R, b, k);
@@ -726,7 +732,7 @@ __device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
 // target u * Z of the inverse CDF and the half slice that owns it.  The draw task goes into the CTA's mailbox:
 // the producer stages that half slice and the consumers find the token.
 template <bool TVO>
-__device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, int b) {
+__device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, int b, int what) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, NR = 2 * K + 1, L = len_of(R, b), T2 = 2 * a.T;
@@ -737,8 +743,8 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
     // lane 0 will need the draw rows' records: asked for now, with everything else
     RowStat sp, sq;
     sp.inv_s = 0.0; sp.e = 0; sp.st = 0; sq = sp;
-    if (lane == 0 && k >= 0) { sp = ld_cg(a.rstat + (int64_t)b * NR + k); if (pair) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k); }
-    if (lane < L && a.o.tv) {
+    if (lane == 0 && k >= 0 && (what & 2)) { sp = ld_cg(a.rstat + (int64_t)b * NR + k); if (pair) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k); }
+    if ((what & 1) && lane < L && a.o.tv) {
         // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
         unsigned long long w = 0;
         for (uint32_t i = 0; i < kSpin; ++i) {
@@ -750,7 +756,7 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         const float z = (float)((double)(w >> 16) * 9.094947017729282e-13);      // 2^-40
         a.o.tv[(int64_t)b * K + lane] = fminf(fmaxf(z, 0.f), 1.f);
     }
-    if (TVO && lane < L && a.s_aux) {
+    if (TVO && (what & 1) && lane < L && a.s_aux) {
         unsigned long long w = 0;
         for (uint32_t i = 0; i < kSpin; ++i) {
             w = __ldcg(a.sacc + (int64_t)b * K + lane);
@@ -760,7 +766,7 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         if ((int)(w & 0xffffull) < T2) atomicExch(a.wait_failed, 1);
         a.s_aux[(int64_t)b * K + lane] = (float)((double)(w >> 16) * 9.094947017729282e-13);
     }
-    if (k < 0) return;
+    if (k < 0 || !(what & 2)) return;
     // the half slices' masses: lanes fetch them in parallel, lane 0 scans them in slice order
     for (int s = lane; s < T2; s += 32) { const DPart dp = load_dpart(a, (int64_t)b * T2 + s); S.d1_tot[s] = dp.tot; S.d1_sq[s] = dp.sq; }
     __syncwarp();
@@ -992,10 +998,15 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
                     red_add_u64(wd, ((unsigned long long)__double2ll_rn(tot * kFixMass) << 4) | 1ull);
                     red_add_u64(wd + 1, ((unsigned long long)__double2ll_rn((double)sq * kFixTv) << 4) | 1ull);
                 }
-                // the sequence's last partial starts the set-up of its draw
-                run_d = atomicAdd(a.p2done + b, 1) == need - 1;
+                // the last partial of the sequence's draw row starts the set-up of its draw, the last partial of all its rows
+                // finishes its TV
+                // (without a TV output the draw row is the sequence's whole second sweep: one counter)
+                const bool all_rows = TVO || a.o.tv != nullptr;
+                if ((flags & 2) && atomicAdd(a.ddone + b, 1) == T2 - 1) run_d |= all_rows ? 2 : 3;
+                if (all_rows && atomicAdd(a.p2done + b, 1) == need - 1) run_d |= 1;
             }
-            if (__shfl_sync(0xffffffffu, run_d, 0)) draw_setup_warp<TVO>(a, S, b);
+            run_d = __shfl_sync(0xffffffffu, run_d, 0);
+            if (run_d) draw_setup_warp<TVO>(a, S, b, run_d);
         }
         // the producer stays until every streaming task has been dealt with here (mailbox entries come first)
         __syncwarp();
@@ -1102,6 +1113,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.wait_failed = wa.ticket + 1;
     wa.p1done = reinterpret_cast<int*>(w + wp.off_p1done);
     wa.p2done = reinterpret_cast<int*>(w + wp.off_p2done);
+    wa.ddone = reinterpret_cast<int*>(w + wp.off_ddone);
     wa.rowcnt = reinterpret_cast<int*>(w + wp.off_rowcnt);
     wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
     wa.rstat = reinterpret_cast<RowStat*>(w + wp.off_rstat);
@@ -1118,18 +1130,6 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
         const long long total = (long long)a.B * (NR * wp.T + (long long)(tv_only ? a.K : (o.tv ? a.K + 1 : 1)) * 2 * wp.T);
         if (total > 0x7fff0000LL) return cudaSuccess;
         wa.ntickets = (int)total;
-        // Distance of the second sweep behind the first, in sequences.  The default is the whole batch (two full
-        // sweeps): measured at the headline shape, a second sweep 24 / 48 / 72 / 96 MB of logits behind the first
-        // found a sixth of its lines in L2 at best, and waited for accept scans more than that saved (0.42 / 0.38 /
-        // 0.35 / 0.30 ms against 0.24 ms).  BEBOP_PIPE_LAG_MB > 0 builds the paired order for experiments.
-        long lag = a.B;
-        if (BEBOP_PIPE_LAG_MB > 0) {
-            const size_t seq_bytes = (size_t)NR * a.nvec * 16;
-            lag = (long)(kLagBytes / (seq_bytes ? seq_bytes : 1));
-            if (lag < 4) lag = 4;
-            if (lag > a.B) lag = a.B;
-        }
-        wa.lag = (int)lag;
     }
     cudaError_t e = cudaMemsetAsync(w, 0, wp.zero_bytes, stream);
     if (e != cudaSuccess) return e;
@@ -1216,7 +1216,7 @@ cudaError_t pipe_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
     wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
-    wa.ntickets = (int)total; wa.lag = a.B;
+    wa.ntickets = (int)total;
     cudaError_t e = cudaMemsetAsync(w, 0, 256, stream);       // ticket counter and wait flag
     if (e != cudaSuccess) return e;
     const int grid = wa.ntickets < grid_max ? wa.ntickets : grid_max;

@@ -49,13 +49,14 @@ struct WaveArgs {
     int* wait_failed;     // [1]
     int* p1done;          // [B] rows of the sequence merged
     int* p2done;          // [B] partials of the sequence's second sweep delivered
+    int* ddone;           // [B] ... of them, partials of the row the sequence's token is drawn from
     int* rowcnt;          // [B][2K+1] pipelined kernel: softmax partials delivered per row
     P1Part* part;         // [B][2K+1][T]
     RowStat* rstat;       // [B][2K+1]
     unsigned long long* dacc;    // [B][2T][2] draw-row mass (2^-58) and sum of squares (2^-40), each << 4 | parts added
     unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
-    int ntickets, lag;               // distance (sequences) of P2 behind P1
+    int ntickets;
     int tv_only;                     // bebop_tv: row pairs only (no bonus row, no accept test, no draw)
     float* s_aux;                    // tv_only: [B] sum of q over the tokens with q <= p, or nullptr
     unsigned long long* sacc;        // [B][K] that sum in 2^-40 units << 16 | parts added
