@@ -32,21 +32,30 @@ namespace bebop {
 
 #ifdef BEBOP_TRACE
 // timeline of the kernel: [2i] earliest, [2i+1] latest global-timer stamp of event i over all CTAs
-__device__ unsigned long long g_pipe_trace[32];
+__device__ unsigned long long g_pipe_trace[64];
 __device__ __forceinline__ void pt_log(int i) {
     unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     atomicMin(&g_pipe_trace[2 * i], t); atomicMax(&g_pipe_trace[2 * i + 1], t);
 }
 #define PTLOG(i) pt_log(i)
+// histogram of an event's time since the kernel's first stamp, 16 buckets of 16.4 us
+__device__ __forceinline__ void pt_hist(int h) {
+    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const unsigned long long t0 = *(volatile unsigned long long*)&g_pipe_trace[0];
+    const unsigned long long k = (t - t0) >> 14;
+    atomicAdd(&g_pipe_trace[16 + 16 * h + (k < 15 ? (int)k : 15)], 1ull);
+}
+#define PTHIST(h) pt_hist(h)
 extern "C" void bebop_debug_pipe_trace(unsigned long long* host32, int reset) {
     if (reset) {
-        unsigned long long init[32];
-        for (int i = 0; i < 16; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
+        unsigned long long init[64];
+        for (int i = 0; i < 32; ++i) { init[2 * i] = i < 8 ? ~0ull : 0ull; init[2 * i + 1] = 0ull; }      // [16..63]: three histograms
         cudaMemcpyToSymbol(g_pipe_trace, init, sizeof(init));
-    } else cudaMemcpyFromSymbol(host32, g_pipe_trace, 32 * sizeof(unsigned long long));
+    } else cudaMemcpyFromSymbol(host32, g_pipe_trace, 64 * sizeof(unsigned long long));
 }
 #else
 #define PTLOG(i) do { } while (0)
+#define PTHIST(h) do { } while (0)
 #endif
 
 namespace {
@@ -767,6 +776,7 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         a.s_aux[(int64_t)b * K + lane] = (float)((double)(w >> 16) * 9.094947017729282e-13);
     }
     if (k < 0 || !(what & 2)) return;
+    if (lane == 0) PTHIST(2);
     // the half slices' masses: lanes fetch them in parallel, lane 0 scans them in slice order
     for (int s = lane; s < T2; s += 32) { const DPart dp = load_dpart(a, (int64_t)b * T2 + s); S.d1_tot[s] = dp.tot; S.d1_sq[s] = dp.sq; }
     __syncwarp();
@@ -1048,9 +1058,9 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
         if (MODE == kModeGreedy) pipe_g<DT>(a, S, d, sd, stage);
         else if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
-        else if (d.phase == 2) { if (tid == 0) PTLOG(7); pipe_p2<DT, MODE == kModeTv>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
+        else if (d.phase == 2) { if (tid == 0) { PTLOG(7); if (d.flags & 2) PTHIST(1); } pipe_p2<DT, MODE == kModeTv>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
         else {
-            if (tid == 0) PTLOG(2);
+            if (tid == 0) { PTLOG(2); PTHIST(0); }
             pipe_d<DT>(a, S, d, sd);
             BEBOP_CTA_SYNC();
             if (tid == 0) PTLOG(3);
