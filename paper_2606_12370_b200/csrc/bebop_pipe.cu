@@ -1,12 +1,15 @@
 // Pipelined kernel: the hot path of bebop_verify as one persistent, ticket-scheduled kernel with the
 // data movement and the bookkeeping taken off the compute warps.
 //
-// The work is a queue of tickets in two blocks: P1 (softmax partial of one slice of one row) for
-// every row, then P2 (TV and residual mass of one half slice of a row pair) for every position;
-// sequences ascending.  Phase A -- merging a row's partials, and the accept scan of a sequence -- has no
-// tickets: it runs in the publisher warp that completes the row / the sequence, long before the second
-// sweep asks for its results.  Nor has the draw: the publisher warp that completes a sequence's second
-// sweep sets the draw up and hands it to its own CTA as a task D (the fast draw with its certificate).
+// The work is a queue of tickets in three blocks, sequences ascending in each: P1 (softmax partial of one
+// slice of one row) for every row; then P2 (TV part and residual mass of one half slice of a row pair) for the
+// row each sequence's token is drawn from; then P2 for the other positions, which only TV needs.  Phase A --
+// merging a row's partials, and the accept scan of a sequence -- has no tickets: it runs in the publisher warp
+// that completes the row / the sequence, long before the second sweep asks for its results.  Nor has the draw:
+// the publisher warp that completes a sequence's draw row sets the draw up and hands it to its own CTA as a
+// task D (the fast draw with its certificate); the one that completes all the sequence's rows writes its TV.
+// A sequence whose fast draw is not certified is listed for the fp64 re-draw kernel, which runs beside the end
+// of this one.
 //
 // A CTA is eight consumer warps, a producer warp and a publisher warp around a ring of shared-memory
 // stages.  The producer's first lane claims tickets, decodes them into runs of consecutive slices,
