@@ -20,9 +20,11 @@ FLAG_MARGIN = 1e-5  # a draw whose accept or CDF margin is below this is "flagge
 
 
 def lib():
+    """The oracle library.  BEBOP_ORACLE_LIB (a path) replaces it: the mutation test points it at deliberately
+    broken builds to show that the pins notice."""
     global _lib
     if _lib is None:
-        _lib = C.CDLL(_build())
+        _lib = C.CDLL(os.environ.get("BEBOP_ORACLE_LIB") or _build())
         _lib.oracle_num_threads.restype = C.c_int
     return _lib
 

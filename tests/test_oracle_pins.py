@@ -74,13 +74,83 @@ def test_tv_special_cases():
     a[:50] = -np.inf; b[50:] = -np.inf
     o = oracle.tv(a[None], b[None])
     assert abs(o["tv"][0] - 1.0) < 1e-15 and o["row_status"][0] == 0
-    # s_aux = sum q 1[q <= p] against a direct numpy evaluation
+
+
+def test_restated_formulas_agree():
+    """The same expressions typed again in numpy.  This guards against typos only: it pins nothing (a formula
+    restated is still the same formula), and the mutation test does not count it."""
+    z = (RNG.standard_normal(100)).astype(np.float32)
     zq = (z + RNG.standard_normal(100)).astype(np.float32)
     o = oracle.tv(z[None], zq[None], temperature_all=0.8)
     p = scipy.special.softmax(z.astype(np.float64) / np.float64(np.float32(0.8)))
     q = scipy.special.softmax(zq.astype(np.float64) / np.float64(np.float32(0.8)))
     assert abs(o["s_aux"][0] - q[q <= p].sum()) < 1e-13
     assert abs(o["tv"][0] - np.maximum(p - q, 0).sum()) < 1e-13
+
+
+def test_s_aux_is_the_scalar_of_the_tv_gradient():
+    """Eq. tv_grad (App. A): d TV / d z_j = -q_j (1[q_j <= p_j] - S) / tau for a draft logit z_j, with S the
+    oracle's s_aux.  The left side is a central finite difference of the oracle's own TV, so a wrong S (summed over
+    the wrong set, or p in place of q) shows as a wrong gradient in every coordinate."""
+    rng = np.random.default_rng(99)
+    h = 2.0 ** -12
+    for V, tau in [(8, 1.0), (32, 0.7), (17, 1.3), (32, 0.5)]:
+        # logits on a grid of 2^-12, so that z +- h is exact in float32
+        zp = (rng.integers(-8192, 8192, V) * h).astype(np.float32)
+        zq = (zp.astype(np.float64) + rng.integers(-4096, 4096, V) * h).astype(np.float32)
+        taud = np.float64(np.float32(tau))
+        base = oracle.tv(zp[None], zq[None], temperature_all=tau)
+        p, _ = oracle.softmax(zp, taud)
+        q, _ = oracle.softmax(zq, taud)
+        assert np.abs(p - q).min() > 1e-4 * q.min()          # no coordinate sits on the kink q = p
+        S = base["s_aux"][0]
+        plus = np.repeat(zq[None], V, 0); minus = plus.copy()
+        plus[np.arange(V), np.arange(V)] += np.float32(h)
+        minus[np.arange(V), np.arange(V)] -= np.float32(h)
+        tgt = np.repeat(zp[None], V, 0)
+        fd = (oracle.tv(tgt, plus, temperature_all=tau)["tv"] - oracle.tv(tgt, minus, temperature_all=tau)["tv"]) / (2 * h)
+        want = -q * ((q <= p).astype(np.float64) - S) / taud
+        np.testing.assert_allclose(fd, want, rtol=0, atol=1e-7)
+        # Prop. 3: the gradient of every coordinate is bounded by q_j / tau
+        assert (np.abs(fd) <= q / taud + 1e-7).all()
+
+
+def _frac(tok):
+    return None if tok == "*" else float(Fraction(tok))
+
+
+def test_golden_dyadic_s_aux_and_margins():
+    """tests/golden/dyadic_margins.txt: S of Eq. tv_grad, the accept margin, both CDF margins and the flag on a
+    four-token case worked out by hand, including a draw that must be flagged and one that must not."""
+    rows, scal, cases = {}, {}, []
+    for line in open(os.path.join(GOLDEN, "dyadic_margins.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        if f[0] == "case":
+            cases.append(f[1:])
+        elif len(f) == 5:
+            rows[f[0]] = [Fraction(x) for x in f[1:]]
+        else:
+            scal[f[0]] = float(Fraction(f[1]))
+    z = {k: np.log2(np.array([float(x) for x in v])).astype(np.float32) for k, v in rows.items()}
+    tau = 1.0 / np.log(2.0)
+    o = oracle.tv(z["p"][None], z["q"][None], temperature_all=tau)
+    assert abs(o["tv"][0] - scal["tv"]) < 1e-6 and abs(o["s_aux"][0] - scal["s_aux"]) < 1e-6
+    tgt = np.stack([z["p"], z["bonus"]])[None]
+    for name, tok, ua, uf, n, y, m_acc, m_cdf, m_cdf_t, flagged in cases:
+        r = oracle.verify(tgt, z["q"][None, None], np.array([[int(tok)]], np.int32),
+                          np.array([[_frac(ua)]], np.float32), np.array([_frac(uf)], np.float32), temperature_all=tau)
+        assert abs(r["tv"][0, 0] - scal["tv"]) < 1e-6, name          # per-position TV of the verify call itself
+        if n != "*":
+            assert r["accept_len"][0] == int(n), name
+        if y != "*":
+            assert r["out_tokens"][0, r["accept_len"][0]] == int(y), name
+        for key, want in (("margin_acc", m_acc), ("margin_cdf", m_cdf), ("margin_cdf_t", m_cdf_t)):
+            if want != "*":
+                got = r[key][0, 0] if key == "margin_acc" else r[key][0]
+                assert abs(got - _frac(want)) < 2e-6, (name, key, got, want)
+        assert bool(r["flagged"][0]) == bool(int(flagged)), name
 
 
 def test_golden_rank_swap_example():
