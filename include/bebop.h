@@ -124,9 +124,10 @@ bebop_status_t bebop_tv(
  * partials of the sweep kept in a scratch array that is part of the library image
  * (BEBOP_TV_STATIC_SCRATCH_BYTES = 1 MiB, one copy per device).  The call allocates nothing and
  * frees nothing.
- *   - Limit: 24 bytes per (row pair, slice) must fit the array, which holds up to 43,690 of them.
- *     Rows are cut into fewer slices as N grows (32 for a handful of long rows, 1 beyond a few
- *     thousand rows), so N up to a few thousand always fits and N > 43,690 never does.  A shape
+ *   - Limit: 16 + 8 bytes per (row pair, slice), in two arrays that each start on a 256-byte boundary, must fit
+ *     the array: up to 43,680 (row pair, slice) entries.  Rows are cut into fewer slices as N grows (32 for a
+ *     handful of long rows, 1 beyond a few thousand rows), so N up to a few thousand always fits and
+ *     N > 43,680 never does.  A shape
  *     that does not fit returns BEBOP_ERR_STATIC_SCRATCH before any launch; use bebop_tv with a
  *     caller workspace then.
  *   - Set-up: the first call on each device looks up the device address of the array
@@ -159,23 +160,29 @@ bebop_status_t bebop_greedy_verify(
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Test and measurement hooks (no counterpart in the paper).
+ * Test and measurement hooks (no counterpart in the paper).  They set process-wide switches that every later
+ * call in the process sees: not thread-safe, and not meant for code that serves requests.
  * bebop_debug_force_general_path(1) makes bebop_verify, bebop_tv and bebop_greedy_verify use the
- * split-row general kernels even for shapes the pipelined kernel takes (process-wide switch; 0 restores).
+ * split-row general kernels even for shapes the pipelined kernel takes (0 restores the default).
  * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
  * shape, of an int32 that after a bebop_verify call holds the number of sequences
  * whose draw was re-done by the fp64 kernels.
  * bebop_debug_set_timing_events(start, stop): two cudaEvent_t handles that the next
  * bebop_verify calls record around the pipelined kernel, on the caller's stream (NULL,
  * NULL switches it off).
- * bebop_debug_set_trace(buf): in builds compiled with -DBEBOP_TRACE, a device buffer of
- * int64 that the pipelined kernel fills with cycle counts (NULL: off); a
- * no-op in normal builds.
+ * bebop_debug_expire_wait(which): the next call's device-side wait number `which` (1: the re-draw kernel's wait
+ * for the list of sequences; 2: the pipelined kernel's wait for a sequence's accept scan) gives up at once, as if
+ * its bound had run out: the call still returns, every row_status carries BEBOP_ROW_WAIT_EXPIRED, and the call
+ * after it is normal again (0: off).  For the test of the bounded waits; nothing is trapped or hung.
+ * bebop_debug_set_draw_kappa(kappa): the factor in the error bound that decides whether bebop_verify keeps a token
+ * drawn from the fp32 prefix sums or re-draws it in double (built-in value 4; a negative argument restores it;
+ * 0 keeps every fp32 draw).  For the test that shows how much room the built-in value leaves.
  */
 void bebop_debug_force_general_path(int on);
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
 void bebop_debug_set_timing_events(void* start, void* stop);
-void bebop_debug_set_trace(void* device_buffer);
+void bebop_debug_expire_wait(int which);
+void bebop_debug_set_draw_kappa(float kappa);
 
 /* Static, host-side, human-readable name of a status code. */
 const char* bebop_status_string(bebop_status_t status);

@@ -51,6 +51,10 @@ def load_library():
     lib.bebop_debug_force_general_path.argtypes = [i32]
     lib.bebop_debug_set_timing_events.restype = None
     lib.bebop_debug_set_timing_events.argtypes = [vp, vp]
+    lib.bebop_debug_set_draw_kappa.restype = None
+    lib.bebop_debug_set_draw_kappa.argtypes = [f32]
+    lib.bebop_debug_expire_wait.restype = None
+    lib.bebop_debug_expire_wait.argtypes = [i32]
     lib.bebop_debug_fallback_offset.restype = sz
     lib.bebop_debug_fallback_offset.argtypes = [i32, i32, i32, i32]
     lib.bebop_status_string.restype = C.c_char_p
@@ -93,6 +97,16 @@ def _rows(t: torch.Tensor, ndim: int):
 
 def bebop_debug_force_general_path(on) -> None:
     load_library().bebop_debug_force_general_path(int(on))
+
+
+def bebop_debug_set_draw_kappa(kappa) -> None:
+    """Factor of the fast draw's error bound (built-in 4; negative restores it; 0 keeps every fp32 draw)."""
+    load_library().bebop_debug_set_draw_kappa(float(kappa))
+
+
+def bebop_debug_expire_wait(which) -> None:
+    """The next call lets device-side wait `which` (1: re-draw list, 2: accept scan) give up at once; 0 = off."""
+    load_library().bebop_debug_expire_wait(int(which))
 
 
 def bebop_debug_set_timing_events(start, stop) -> None:
@@ -176,7 +190,7 @@ def bebop_verify(target_logits, draft_logits, draft_tokens, u_accept, u_final, d
 
 
 def bebop_tv(target_logits, draft_logits, temperature=None, temperature_all=1.0, workspace=None,
-             want_s_aux=True):
+             want_s_aux=True, want_status=True):
     """TV distance (and the auxiliary S) of N paired rows [N,V]."""
     lib = load_library()
     N, V = target_logits.shape
@@ -187,7 +201,7 @@ def bebop_tv(target_logits, draft_logits, temperature=None, temperature_all=1.0,
     dp, ldd = _rows(draft_logits, 2)
     tv = _new(N, torch.float32, dev)
     s_aux = _new(N, torch.float32, dev) if want_s_aux else None
-    st = _new(N, torch.int32, dev)
+    st = _new(N, torch.int32, dev) if want_status else None
     ws, wsb = _workspace(N, 1, V, dt, dev, workspace)
     _check(lib.bebop_tv(tp, ldt, dp, ldd, _ptr(temperature), float(temperature_all), N, V, dt,
                         _ptr(tv), _ptr(s_aux), _ptr(st), _ptr(ws), wsb, _stream()))

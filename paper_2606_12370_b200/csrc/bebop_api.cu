@@ -11,11 +11,16 @@ namespace {
 // kernel applies, so that both paths are covered by the parity tests.
 int g_path = 0;   // 0: pipelined kernel where it applies, else the general kernels; 1: general kernels only
 
+int g_expire_wait = 0;   // test hook: which device-side wait the next call lets give up at once
+float g_draw_kappa = -1.f;   // test hook: factor of the fast draw's error bound (negative: the built-in value)
+
 // Built-in scratch of bebop_tv_static: one array per device the module is loaded on.  Nothing in it
 // has to start at zero (every partial is written before it is read).
 static __device__ __align__(256) unsigned char g_tv_scratch[BEBOP_TV_STATIC_SCRATCH_BYTES];
 constexpr int kMaxDevices = 64;
-void* g_tv_scratch_ptr[kMaxDevices] = {nullptr};   // device address of g_tv_scratch, looked up once per device
+// device address of g_tv_scratch, looked up once per device.  A plain host cache: two threads that make a device's
+// first call at the same time both look the address up and store the same value.
+void* g_tv_scratch_ptr[kMaxDevices] = {nullptr};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -67,6 +72,11 @@ RowArgs row_args(const void* target, int64_t ld_t, const void* draft, int64_t ld
 }
 
 }  // namespace
+
+namespace bebop {
+int take_expire_wait() { const int w = g_expire_wait; g_expire_wait = 0; return w; }
+float draw_kappa() { return g_draw_kappa >= 0.f ? g_draw_kappa : 4.0f; }
+}  // namespace bebop
 
 extern "C" {
 
@@ -195,13 +205,15 @@ bebop_status_t bebop_tv_static(const void* target_logits, int64_t ld_target, con
 
 void bebop_debug_force_general_path(int on) { g_path = on; }
 
-void bebop_debug_set_trace(void* p) { wave_set_trace(static_cast<long long*>(p)); }
+void bebop_debug_expire_wait(int which) { g_expire_wait = which; }
 
-void bebop_debug_set_timing_events(void* start, void* stop) { wave_set_events(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop)); }
+void bebop_debug_set_draw_kappa(float kappa) { g_draw_kappa = kappa; }
+
+void bebop_debug_set_timing_events(void* start, void* stop) { pipe_set_events(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop)); }
 
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt) {
     if (check_shape(B, K, V, dt) != BEBOP_OK) return 0;
-    return make_plan(B, K, V, (int)dt).off_wave + kFbCountOffset;
+    return make_plan(B, K, V, (int)dt).off_pipe + kFbCountOffset;
 }
 
 const char* bebop_status_string(bebop_status_t status) {

@@ -41,19 +41,22 @@ cudaError_t general_greedy(const RowArgs& a, const Plan& p, const int32_t* draft
                            int32_t* accept_len, int32_t* out_tokens, int32_t* row_status, char* ws,
                            cudaStream_t stream);
 
-void wave_set_trace(long long* p);                            // trace buffer of the main kernel (BEBOP_TRACE builds)
-void wave_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the main kernel of the next calls (nullptr: off)
+// Test hook: the number of the device-side wait that the next call lets give up at once (0: none); reading it clears it.
+int take_expire_wait();
+// Test hook: the factor of the fast draw's error bound (4 unless a test has set another value).
+float draw_kappa();
+void pipe_set_events(cudaEvent_t start, cudaEvent_t stop);   // bracket the main kernel of the next calls (nullptr: off)
 
-// fp64 re-draw of the sequences a kernel listed (bebop_redraw.cu); `w` is the wave workspace laid out by `wp`.
+// fp64 re-draw of the sequences a kernel listed (bebop_redraw.cu); `w` is the pipelined kernel's workspace laid out by `wp`.
 // Launched behind the pipelined kernel, it follows the list while that kernel still runs: the low half of
 // `fb_count` is the number of listed sequences so far, the high half the number of sequences whose draw is
 // decided, `expect` of them in all.  It also turns a device-side wait that gave up (`wait_failed`) into status
 // bit ST_WAIT of every row.
 cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const unsigned long long* fb_count,
                           const FbRec* fb_list, int expect, int* wait_failed, char* w,
-                          const WavePlan& wp, cudaStream_t stream);
+                          const PipePlan& wp, cudaStream_t stream, bool expire_list_wait = false);
 
-// Pipelined kernel (bebop_pipe.cu): the wave schedule with a producer warp that stages every task's
+// Pipelined kernel (bebop_pipe.cu): a ticket schedule with a producer warp that stages every task's
 // logits in shared memory by bulk copies while the other warps compute; same contract.  With `tv_only` it is
 // bebop_tv: B row pairs (K = 1), o.tv and s_aux the outputs, no tokens, no uniforms, no draw.
 bool pipe_supported(const RowArgs& a);

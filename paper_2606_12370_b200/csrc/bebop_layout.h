@@ -7,24 +7,18 @@
 namespace bebop {
 
 // Workspace of the pipelined kernel and of the fp64 re-draw kernels.
-#ifndef BEBOP_PIPE_SLICE_VECS
-#define BEBOP_PIPE_SLICE_VECS 2048
-#endif
-constexpr int kPipeSliceVecs = BEBOP_PIPE_SLICE_VECS;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
+constexpr int kPipeSliceVecs = 2048;   // 16-byte vectors per row slice, at most: one stage of the kernel's ring
 // A sequence whose draw goes to the fp64 re-draw: all the re-draw kernels need to find its rows.
 struct alignas(16) FbRec {
     int b1;                             // sequence + 1 (0: the record is not written yet)
     int kp;                             // 2 * draw row + (1 if the row is a residual of a target / draft pair)
     int ep, eq;                         // reference exponents of the target row and of the draft row
 };
-#ifndef BEBOP_REDRAW_CUT
-#define BEBOP_REDRAW_CUT 4
-#endif
-constexpr int kRedrawCut = BEBOP_REDRAW_CUT;   // the fp64 re-draw cuts every row slice into so many work items
+constexpr int kRedrawCut = 4;   // the fp64 re-draw cuts every row slice into so many work items
 constexpr size_t kRedrawTicketOffset = 192;   // unsigned: next work item of the fp64 re-draw (zeroed head of the workspace)
 constexpr size_t kFbCountOffset = 128;   // 8 bytes inside the zeroed head of the workspace: low int, sequences listed for the fp64
                                          // re-draw; high int, sequences whose draw is decided
-struct WavePlan {
+struct PipePlan {
     int T, slice_vecs;     // slices per row, vectors per slice (multiple of 16)
     size_t off_p1done, off_p2done, off_ddone, off_xdone, off_xsdone, off_fbrec, off_rowcnt, zero_bytes;
     size_t off_xsum, off_xmass;   // fp64 re-draw: per listed sequence done counter; sums and masses per quarter slice
@@ -45,14 +39,14 @@ struct Plan {
     size_t off_dstats;  // double2[B][2][nsplit_d]       (m, S) partials, fp64
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
-    size_t off_wave;    // workspace of the pipelined kernel
+    size_t off_pipe;    // workspace of the pipelined kernel
     size_t total;
 };
 
 
-static inline WavePlan make_wave_plan(int B, int K, int nvec, int dt, int slice_cap = kPipeSliceVecs) {
+static inline PipePlan make_pipe_plan(int B, int K, int nvec, int dt, int slice_cap = kPipeSliceVecs) {
     (void)dt;
-    WavePlan w;
+    PipePlan w;
     w.T = (nvec + slice_cap - 1) / slice_cap; if (w.T < 1) w.T = 1;
     w.slice_vecs = (((nvec + w.T - 1) / w.T) + 15) & ~15;   // halves (phase P2) stay 128-byte aligned
     const size_t NR = (size_t)(2 * K + 1);
@@ -105,7 +99,7 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     {
-        p.off_wave = o;   o = align256(o + make_wave_plan(B, K, p.nvec, dt).total);
+        p.off_pipe = o;   o = align256(o + make_pipe_plan(B, K, p.nvec, dt).total);
     }
     p.total = o;
     return p;

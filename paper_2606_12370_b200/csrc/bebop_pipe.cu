@@ -28,72 +28,25 @@
 //
 // Every wait is bounded; a wait that gives up sets the wait flag (status bit 32 of every row).
 // No multicast, no cluster: each CTA copies from this GPU's own memory.
-#define BEBOP_CTA_SYNC() asm volatile("bar.sync 1, 256;" ::: "memory")
 #include "bebop_pipe.cuh"
 
 namespace bebop {
 
-#ifdef BEBOP_TRACE
-// timeline of the kernel: [2i] earliest, [2i+1] latest global-timer stamp of event i over all CTAs
-__device__ unsigned long long g_pipe_trace[64];
-__device__ __forceinline__ void pt_log(int i) {
-    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    atomicMin(&g_pipe_trace[2 * i], t); atomicMax(&g_pipe_trace[2 * i + 1], t);
-}
-#define PTLOG(i) pt_log(i)
-// histogram of an event's time since the kernel's first stamp, 16 buckets of 16.4 us
-__device__ __forceinline__ void pt_hist(int h) {
-    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    const unsigned long long t0 = *(volatile unsigned long long*)&g_pipe_trace[0];
-    const unsigned long long k = (t - t0) >> 14;
-    atomicAdd(&g_pipe_trace[16 + 16 * h + (k < 15 ? (int)k : 15)], 1ull);
-}
-#define PTHIST(h) pt_hist(h)
-extern "C" void bebop_debug_pipe_trace(unsigned long long* host32, int reset) {
-    if (reset) {
-        unsigned long long init[64];
-        for (int i = 0; i < 32; ++i) { init[2 * i] = i < 8 ? ~0ull : 0ull; init[2 * i + 1] = 0ull; }      // [16..63]: three histograms
-        cudaMemcpyToSymbol(g_pipe_trace, init, sizeof(init));
-    } else cudaMemcpyFromSymbol(host32, g_pipe_trace, 64 * sizeof(unsigned long long));
-}
-#else
-#define PTLOG(i) do { } while (0)
-#define PTHIST(h) do { } while (0)
-#endif
-
 namespace {
 
-#ifndef BEBOP_PIPE_STAGES
-#define BEBOP_PIPE_STAGES 2
-#endif
-#ifndef BEBOP_PIPE_CTAS
-#define BEBOP_PIPE_CTAS 3
-#endif
 // what the kernel is compiled for: bebop_verify; bebop_tv (row pairs, no accept test, no draw); the greedy mode
 // (one sweep over the target rows for their argmax)
 constexpr int kModeVerify = 0, kModeTv = 1, kModeGreedy = 2;
-constexpr int NST = BEBOP_PIPE_STAGES;            // stages of the ring
-constexpr int PIPE_CTAS = BEBOP_PIPE_CTAS;        // CTAs per SM the kernel is built for
+constexpr int NST = 2;                            // stages of the ring
+constexpr int PIPE_CTAS = 3;                      // CTAs per SM the kernel is built for
 constexpr int PC = WT;                            // consumer threads (8 warps); thread PC is the producer
 constexpr int PT = PC + 64;                       // + producer warp + publisher warp
 constexpr int PSLICE = kPipeSliceVecs;            // vectors per stage
 constexpr int STAGE_BYTES = PSLICE * 16;
-#ifndef BEBOP_PIPE_NOHINT
-#define BEBOP_PIPE_NOHINT 0
-#endif
 constexpr int kPend = 4;                          // runs a producer may set aside
-#ifndef BEBOP_PIPE_BATCH
-#define BEBOP_PIPE_BATCH 5
-#endif
-#ifndef BEBOP_PIPE_TAIL
-#define BEBOP_PIPE_TAIL 8
-#endif
-constexpr int kTailZone = BEBOP_PIPE_TAIL;        // the last kTailZone tickets per CTA are claimed kBatchTail at a time
-#ifndef BEBOP_PIPE_BATCH_TAIL
-#define BEBOP_PIPE_BATCH_TAIL 2
-#endif
-constexpr int kBatchTail = BEBOP_PIPE_BATCH_TAIL;
-constexpr int kBatch = BEBOP_PIPE_BATCH;          // tickets claimed at a time (measured: 4 to 6 alike, 2 and 8 slower)
+constexpr int kTailZone = 8;                      // the last kTailZone tickets per CTA are claimed kBatchTail at a time
+constexpr int kBatchTail = 2;
+constexpr int kBatch = 5;                         // tickets claimed at a time (measured: 4 to 6 alike, 2 and 8 slower)
 constexpr double kFixTv = 1099511627776.0;             // 2^40: fixed point of TV parts and sums of squares
 constexpr double kFixMass = 288230376151711744.0;      // 2^58: fixed point of the draw-row mass
 constexpr uint32_t kBarSpin = 1u << 20;           // tries of one barrier wait (each try itself waits a while)
@@ -121,15 +74,16 @@ struct DrawTask {
     RowScale P, Q;
 };
 constexpr int kMbox = 16;                    // mailbox entries: more than the tasks a CTA can have unpublished
-static_assert(kMbox >= BEBOP_PIPE_BATCH + BEBOP_PIPE_STAGES + 1, "a run's tasks plus the ring may each complete a sequence before the producer looks");
+static_assert(kMbox >= kBatch + NST + 1, "a run's tasks plus the ring may each complete a sequence before the producer looks");
 
-struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of one (phase, wave) block from offset off
+struct Run { int ph, wv, off, cnt; };       // cnt consecutive tasks of sequence wv in phase ph, from offset off
 
 struct PipeShared {
-    WaveShared W;                               // scratch of phases A and D
+    DrawShared W;                               // scratch of phases A and D
     TaskDesc desc[NST];
     unsigned long long full[NST], empty[NST];   // mbarriers: data and description there / stage free again
     unsigned long long pdone[NST];              // mbarrier: the eight warp partials of the stage's task are there
+    unsigned long long dsync;                   // mbarrier: the consumer warps meet here inside a draw task (bounded wait)
     float wf[NST][2][WW];                       // per-warp partials of the task in the stage
     double wd[NST][WW];
     int wi[NST][WW];
@@ -140,7 +94,6 @@ struct PipeShared {
     float vsum[PSLICE / 2];                     // D: residual mass per vector of the half slice
     double d1_tot[2 * MAX_SLICES];              // publisher: half-slice masses and sums of squares of a sequence
     float d1_sq[2 * MAX_SLICES];
-    int logn;                                   // trace builds: events logged
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -172,8 +125,7 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 }
 __device__ __forceinline__ unsigned long long l2_policy(bool keep) {
     unsigned long long p;
-    if (BEBOP_PIPE_NOHINT) asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
-    else if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
     else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
@@ -186,14 +138,16 @@ __device__ __forceinline__ int div_by(int n, int d, double inv) {
     return q;
 }
 __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
+// The consumer warps of a CTA meet (inside a draw task).  A counted barrier with a bounded wait, not bar.sync: should
+// a warp have left the loop after a wait of its own gave up, the others still return, with the wait flag set.
+// `phase` is the warp's count of such meetings so far (every consumer warp sees the same draw tasks).
+__device__ __forceinline__ void consumers_meet(int* wait_failed, unsigned long long* bar, uint32_t& phase) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+    if (!mbar_wait(bar, phase & 1u)) atomicExch(wait_failed, 1);
+    ++phase;
+}
 
-
-#ifdef BEBOP_TRACE
-// event log of one CTA: (clock, code * 1e6 + task number)
-#define PLOG(code, n) do { if (blockIdx.x == 5 && a.trace) { const int k_ = atomicAdd(&S.logn, 1); if (k_ < 3000) { a.trace[2048 + 2 * k_] = clock64(); a.trace[2049 + 2 * k_] = (long long)(code) * 1000000 + (n); } } } while (0)
-#else
-#define PLOG(code, n) do { } while (0)
-#endif
 
 // ------------------------------------------------------------------ producer
 // One thread.  Tickets are claimed kBatch at a time; consecutive tickets of one (phase, sequence) block are
@@ -203,7 +157,7 @@ __device__ __forceinline__ uint4 lds16(const unsigned char* p) { return *reinter
 // when it has delivered the last partial of a sequence's second sweep, and the producer stages it ahead of
 // the next ticket.  Returns when the stop description has been handed to the consumers.
 template <int DT, int MODE>
-__device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsigned char* data) {
+__device__ __forceinline__ void producer(const PipeArgs& a, PipeShared& S, unsigned char* data) {
     constexpr bool TVO = MODE == kModeTv, GRD = MODE == kModeGreedy;
     const RowArgs& R = a.r;
     const int K = R.K, T = a.T, T2 = 2 * a.T, NR = 2 * K + 1;
@@ -255,6 +209,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     // the sequence's record of the accept scan, valid once its mark is set (waits, bounded, if asked to)
     auto seq_info = [&](int b, bool wait) {
         SeqInfo si = ld_cg(a.sinfo + b);
+        if (a.expire) { if (wait) si.pad = 0; return si; }          // test hook: this wait's bound has run out already
         if (wait) for (uint32_t i = 0; si.pad == 0 && i < kSpin; ++i) { __nanosleep(64); si = ld_cg(a.sinfo + b); }
         return si;
     };
@@ -263,6 +218,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
     auto ready = [&](int ph, int b, bool wait) {
         if (ph != 2) return true;
         if (seen_b == b) return true;
+        if (a.expire && !wait) return false;                        // test hook: every second-sweep run goes through the wait
         const SeqInfo si = seq_info(b, wait);
         if (si.pad == 0) return false;
         seen = si; seen_b = b;
@@ -274,7 +230,6 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
         const int stage = it % NST;
         if (!mbar_wait(&S.empty[stage], ((uint32_t)(it / NST) & 1u) ^ 1u)) atomicExch(a.wait_failed, 1);
         S.desc[stage] = d;
-        PLOG(1 + 10 * d.phase, it);
         const uint32_t bytes = (uint32_t)d.nv * 16u;
         if (row0 && bytes) {
             mbar_arrive_expect(&S.full[stage], row1 ? 2u * bytes : bytes);
@@ -319,7 +274,7 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
                 const int cnt = (a.ntickets - last_seen <= tail_zone) ? kBatchTail : kBatch;
                 bt = atomicAdd(a.ticket, cnt); bleft = min(cnt, a.ntickets - bt);
                 last_seen = bt;
-                if (bleft <= 0) { bleft = 0; exhausted = true; PTLOG(1); }
+                if (bleft <= 0) { bleft = 0; exhausted = true; }
             }
             if (bleft == 0) {
                 if (npend > 0) continue;
@@ -416,8 +371,8 @@ __device__ __forceinline__ void producer(const WaveArgs& a, PipeShared& S, unsig
 // integer exponents, fp64 sums in a fixed tree) and leaves the row's normaliser; the warp that merges
 // the last row of a SEQUENCE runs the accept scan at once and writes accept_len, the accepted tokens,
 // p(x), q(x), the status and the stop position.  No ticket, no CTA barrier, and the work is done
-// long before phase P2 of the wave is handed out.
-__device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) {
+// long before the second sweep of the sequence is handed out.
+__device__ __forceinline__ void merge_row_warp(const PipeArgs& a, int b, int r) {
     const int lane = threadIdx.x & 31;
     const int NR = 2 * a.r.K + 1, T = a.T;
     const P1Part* pp = a.part + ((int64_t)b * NR + r) * T;
@@ -448,7 +403,7 @@ __device__ __forceinline__ void merge_row_warp(const WaveArgs& a, int b, int r) 
 }
 
 template <int DT, bool TVO>
-__device__ __noinline__ void accept_warp(const WaveArgs& a, int b) {
+__device__ __noinline__ void accept_warp(const PipeArgs& a, int b) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, V = R.V, L = len_of(R, b), NR = 2 * K + 1;
@@ -527,7 +482,7 @@ __device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long
 
 // P1: softmax partial (E, S) of one slice of one row, from shared memory.
 template <int DT>
-__device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+__device__ __forceinline__ void pipe_p1(const PipeArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
                                         int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
     const RowArgs& R = a.r;
@@ -592,7 +547,7 @@ __device__ __forceinline__ void pipe_p1(const WaveArgs& a, PipeShared& S, const 
 
 // Greedy mode: maximum and lowest index of the maximum over one slice of a target row (no exponentials).
 template <int DT>
-__device__ __forceinline__ void pipe_g(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+__device__ __forceinline__ void pipe_g(const PipeArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
                                        int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / PC;
     const RowArgs& R = a.r;
@@ -616,6 +571,7 @@ __device__ __forceinline__ void pipe_g(const WaveArgs& a, PipeShared& S, const T
 #pragma unroll
     for (int u = 1; u < NV; ++u) m = max_nan(m, vec_max<DT>(raw[u]));
     if (!(m < INFINITY)) m = __int_as_float(0x7fc00000);      // NaN or +inf poisons the row
+    m += 0.f;                                                 // -0 becomes +0: the ordered-integer maximum below must not tell them apart
     // the thread's lowest token with that value (its vectors ascend with u)
     int idx = INT_MAX;
     if (m == m && m > -INFINITY) {
@@ -641,7 +597,7 @@ __device__ __forceinline__ void pipe_g(const WaveArgs& a, PipeShared& S, const T
 // also the mass in double and the sum of squares.  Target row in the first half of the stage, draft
 // row in the second.
 template <int DT, bool TVO>
-__device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
+__device__ __forceinline__ void pipe_p2(const PipeArgs& a, PipeShared& S, const TaskDesc& d, const unsigned char* data,
                                         int stage) {
     constexpr int VEC = Elem<DT>::VEC, NV = PSLICE / (2 * PC);
     const RowArgs& R = a.r;
@@ -724,7 +680,7 @@ __device__ __forceinline__ void pipe_p2(const WaveArgs& a, PipeShared& S, const 
 
 // ------------------------------------------------------------------ the draw
 // mass and sum of squares of half slice i of a sequence's draw rows (waits, bounded, for a part not there yet)
-__device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
+__device__ __forceinline__ DPart load_dpart(const PipeArgs& a, int64_t i) {
     unsigned long long w0 = 0, w1 = 0;
     for (uint32_t k = 0; k < kSpin; ++k) {
         w0 = __ldcg(a.dacc + 2 * i); w1 = __ldcg(a.dacc + 2 * i + 1);
@@ -744,7 +700,7 @@ __device__ __forceinline__ DPart load_dpart(const WaveArgs& a, int64_t i) {
 // target u * Z of the inverse CDF and the half slice that owns it.  The draw task goes into the CTA's mailbox:
 // the producer stages that half slice and the consumers find the token.
 template <bool TVO>
-__device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, int b, int what) {
+__device__ __noinline__ void draw_setup_warp(const PipeArgs& a, PipeShared& S, int b, int what) {
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, NR = 2 * K + 1, L = len_of(R, b), T2 = 2 * a.T;
@@ -779,7 +735,6 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
         a.s_aux[(int64_t)b * K + lane] = (float)((double)(w >> 16) * 9.094947017729282e-13);
     }
     if (k < 0 || !(what & 2)) return;
-    if (lane == 0) PTHIST(2);
     // the half slices' masses: lanes fetch them in parallel, lane 0 scans them in slice order
     for (int s = lane; s < T2; s += 32) { const DPart dp = load_dpart(a, (int64_t)b * T2 + s); S.d1_tot[s] = dp.tot; S.d1_sq[s] = dp.sq; }
     __syncwarp();
@@ -811,7 +766,7 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
             if (!room) atomicExch(a.wait_failed, 1);
             else {
                 DrawTask t;
-                t.tt = Tt; t.base = base; t.bound = (float)draw_bound(sumsq); t.c = __int_as_float(si.pad0);
+                t.tt = Tt; t.base = base; t.bound = (float)draw_bound(sumsq, (double)a.kappa); t.c = __int_as_float(si.pad0);
                 t.b = b; t.k = k; t.owner = owner; t.pair = pair ? 1 : 0;
                 t.P = row_scale(sp); t.Q = pair ? row_scale(sq) : no_row();
                 S.mbox[tail % kMbox] = t;
@@ -828,10 +783,10 @@ __device__ __noinline__ void draw_setup_warp(const WaveArgs& a, PipeShared& S, i
 // running sum are further apart than the error bound on both sides of the token; else the sequence is listed
 // for the fp64 re-draw.
 template <int DT>
-__device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const TaskDesc& d, const unsigned char* data) {
+__device__ __forceinline__ void pipe_d(const PipeArgs& a, PipeShared& PS, const TaskDesc& d, const unsigned char* data, uint32_t& meet) {
     constexpr int VEC = Elem<DT>::VEC;
     const RowArgs& R = a.r;
-    WaveShared& S = PS.W;
+    DrawShared& S = PS.W;
     float* vsum = PS.vsum;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = R.K, NR = 2 * K + 1, b = d.b, k = d.r;
@@ -854,7 +809,7 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
             residual_vec<DT, true>(rp, rq, c, SP, SQ, r, nullptr);
             vsum[v] = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
         }
-        BEBOP_CTA_SYNC();
+        consumers_meet(a.wait_failed, &PS.dsync, meet);
         // contiguous ranges of vectors per thread, inclusive scan over threads
         const int per = (nv + PC - 1) / PC;
         const int vb = min(tid * per, nv), ve = min(vb + per, nv);
@@ -864,7 +819,7 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { double t2 = shfl_up_d(incl, o); if (lane >= o) incl += t2; }
         if (lane == 31) S.redd[warp] = incl;
-        BEBOP_CTA_SYNC();
+        consumers_meet(a.wait_failed, &PS.dsync, meet);
         double woff = 0.0;
         for (int w = 0; w < warp; ++w) woff += S.redd[w];
         double prev = shfl_up_d(incl, 1);
@@ -903,9 +858,9 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
     // at most one thread should have found the token
     const unsigned own = __ballot_sync(0xffffffffu, found_y >= 0);
     if (lane == 0) S.redi[warp] = -1;
-    BEBOP_CTA_SYNC();
+    consumers_meet(a.wait_failed, &PS.dsync, meet);
     if (own && lane == (__ffs(own) - 1)) S.redi[warp] = (__popc(own) == 1 && found_cert) ? found_y : -2;
-    BEBOP_CTA_SYNC();
+    consumers_meet(a.wait_failed, &PS.dsync, meet);
     if (tid == 0) {
         int y = -1, cnt = 0;
         for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
@@ -927,7 +882,7 @@ __device__ __forceinline__ void pipe_d(const WaveArgs& a, PipeShared& PS, const 
 // row, whose last merged row starts the accept scan of the sequence; P2 -- the TV part (and the
 // draw-row mass) and the sequence's counter.
 template <int DT, int MODE>
-__device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
+__device__ __forceinline__ void publisher(const PipeArgs& a, PipeShared& S) {
     constexpr bool TVO = MODE == kModeTv, GRD = MODE == kModeGreedy;
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
@@ -1030,7 +985,7 @@ __device__ __forceinline__ void publisher(const WaveArgs& a, PipeShared& S) {
 }  // namespace
 
 template <int DT, int MODE>
-__global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ WaveArgs a) {
+__global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ PipeArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* data = smem;
     PipeShared& S = *reinterpret_cast<PipeShared*>(smem + (size_t)NST * STAGE_BYTES);
@@ -1038,10 +993,10 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
     // the re-draw kernel behind this one may be scheduled as CTAs of this one leave (programmatic dependent
     // launch); it follows the list of sequences as it grows (`fb_count` tells it when the list is complete)
     if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid == 0) PTLOG(0);
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], WW + 1); mbar_init(&S.pdone[i], WW); }
-        S.logn = 0; S.mb_tail = 0; S.mb_head = 0; S.pub_count = 0;
+        mbar_init(&S.dsync, WW);
+        S.mb_tail = 0; S.mb_head = 0; S.pub_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -1051,27 +1006,24 @@ __global__ void __launch_bounds__(PT, PIPE_CTAS) k_pipe(const __grid_constant__ 
         return;
     }
     const int lane = tid & 31;
+    uint32_t meet = 0;
     for (int it = 0;; ++it) {
         const int stage = it % NST;
         const uint32_t par = (uint32_t)(it / NST) & 1u;
         if (!mbar_wait(&S.full[stage], par)) { if (tid == 0) atomicExch(a.wait_failed, 1); break; }
         const TaskDesc d = S.desc[stage];
         if (d.phase < 0) break;
-        if (tid == 0) PLOG(2, it);
         const unsigned char* sd = data + (size_t)stage * STAGE_BYTES;
         if (MODE == kModeGreedy) pipe_g<DT>(a, S, d, sd, stage);
-        else if (d.phase == 0) { pipe_p1<DT>(a, S, d, sd, stage); if (tid == 0) PTLOG(6); }
-        else if (d.phase == 2) { if (tid == 0) { PTLOG(7); if (d.flags & 2) PTHIST(1); } pipe_p2<DT, MODE == kModeTv>(a, S, d, sd, stage); if (tid == 0) PTLOG(5); }
+        else if (d.phase == 0) pipe_p1<DT>(a, S, d, sd, stage);
+        else if (d.phase == 2) pipe_p2<DT, MODE == kModeTv>(a, S, d, sd, stage);
         else {
-            if (tid == 0) { PTLOG(2); PTHIST(0); }
-            pipe_d<DT>(a, S, d, sd);
-            BEBOP_CTA_SYNC();
-            if (tid == 0) PTLOG(3);
+            pipe_d<DT>(a, S, d, sd, meet);
+            consumers_meet(a.wait_failed, &S.dsync, meet);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&S.empty[stage]);
     }
-    if (tid == 0) PTLOG(4);
 }
 
 // -----------------------------------------------------------------------------
@@ -1100,7 +1052,6 @@ int pipe_grid() {
 
 }  // namespace
 
-extern long long* g_wave_trace;
 extern cudaEvent_t g_ev_start, g_ev_stop;
 
 bool pipe_supported(const RowArgs& a) {
@@ -1115,11 +1066,11 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     const int grid_max = tv_only ? (a.dt == 0 ? pipe_grid<0, kModeTv>() : pipe_grid<1, kModeTv>())
                                  : (a.dt == 0 ? pipe_grid<0, kModeVerify>() : pipe_grid<1, kModeVerify>());
     if (grid_max < 1) return cudaSuccess;
-    const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
-    WaveArgs wa;
+    const PipePlan wp = make_pipe_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
+    PipeArgs wa;
     wa.r = a; wa.draft_tokens = draft_tokens; wa.u_accept = u_accept; wa.u_final = u_final; wa.o = o;
     wa.stop = reinterpret_cast<int*>(ws + p.off_stop);
-    char* w = ws + p.off_wave;
+    char* w = ws + p.off_pipe;
     wa.fb_count = reinterpret_cast<unsigned long long*>(w + kFbCountOffset);
     wa.fb_list = reinterpret_cast<FbRec*>(w + wp.off_fbrec);
     wa.ticket = reinterpret_cast<int*>(w);
@@ -1133,10 +1084,12 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     wa.dacc = reinterpret_cast<unsigned long long*>(w + wp.off_dpart);
     wa.tvacc = reinterpret_cast<unsigned long long*>(w + wp.off_tvacc);
     wa.sinfo = reinterpret_cast<SeqInfo*>(w + wp.off_sinfo);
+    const int expire = take_expire_wait();
+    wa.expire = expire == 2 ? 1 : 0;
+    wa.kappa = draw_kappa();
     wa.tv_only = tv_only ? 1 : 0;
     wa.s_aux = tv_only ? s_aux : nullptr;
     wa.sacc = (tv_only && s_aux) ? reinterpret_cast<unsigned long long*>(w + wp.off_sacc) : nullptr;
-    wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
     {
         const long long NR = 2 * a.K + 1;
@@ -1159,7 +1112,7 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
     if (e != cudaSuccess) return e;
     *launched = true;
-    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, tv_only ? 0 : a.B, wa.wait_failed, w, wp, stream);
+    return redraw_launch(a, u_final, o, wa.fb_count, wa.fb_list, tv_only ? 0 : a.B, wa.wait_failed, w, wp, stream, expire == 1);
 }
 
 // ------------------------------------------------------------------ greedy mode
@@ -1167,7 +1120,7 @@ namespace {
 
 // One warp per sequence, behind the sweep: lane k merges the slice records of target row k (maximum, lowest
 // index), then the argmax match x_k == g_k runs down the drafts; the argmax of the stop position is emitted.
-__global__ void __launch_bounds__(128) k_greedy_finish(WaveArgs a, int32_t* __restrict__ accept_len,
+__global__ void __launch_bounds__(128) k_greedy_finish(PipeArgs a, int32_t* __restrict__ accept_len,
                                                         int32_t* __restrict__ out_tokens, int32_t* __restrict__ row_status) {
     asm volatile("griddepcontrol.wait;" ::: "memory");       // programmatic dependent of the sweep
     const RowArgs& R = a.r;
@@ -1218,16 +1171,15 @@ cudaError_t pipe_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_to
     *launched = false;
     const int grid_max = a.dt == 0 ? pipe_grid<0, kModeGreedy>() : pipe_grid<1, kModeGreedy>();
     if (grid_max < 1) return cudaSuccess;
-    const WavePlan wp = make_wave_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
+    const PipePlan wp = make_pipe_plan(a.B, a.K, a.nvec, a.dt, PSLICE);
     const long long total = (long long)a.B * (a.K + 1) * wp.T;
     if (total > 0x7fff0000LL) return cudaSuccess;
-    char* w = ws + p.off_wave;
-    WaveArgs wa = {};
+    char* w = ws + p.off_pipe;
+    PipeArgs wa = {};
     wa.r = a; wa.draft_tokens = draft_tokens;
     wa.ticket = reinterpret_cast<int*>(w);
     wa.wait_failed = wa.ticket + 1;
     wa.part = reinterpret_cast<P1Part*>(w + wp.off_part);
-    wa.trace = g_wave_trace;
     wa.T = wp.T; wa.slice_vecs = wp.slice_vecs;
     wa.ntickets = (int)total;
     cudaError_t e = cudaMemsetAsync(w, 0, 256, stream);       // ticket counter and wait flag

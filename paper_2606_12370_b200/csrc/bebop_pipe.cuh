@@ -34,7 +34,7 @@ struct __align__(16) SeqInfo {          // per sequence, written by phase A
     int pad;
 };
 
-struct WaveArgs {
+struct PipeArgs {
     RowArgs r;
     const int32_t* draft_tokens;
     const float* u_accept;
@@ -57,10 +57,11 @@ struct WaveArgs {
     unsigned long long* tvacc;   // [B][K] TV sum in 2^-40 units << 16 | parts added
     SeqInfo* sinfo;       // [B]
     int ntickets;
+    int expire;                      // test hook: the producers' wait for a sequence's accept scan gives up at once
+    float kappa;                     // factor of the fast draw's error bound (kDrawKappa; a test hook can change it)
     int tv_only;                     // bebop_tv: row pairs only (no bonus row, no accept test, no draw)
     float* s_aux;                    // tv_only: [B] sum of q over the tokens with q <= p, or nullptr
     unsigned long long* sacc;        // [B][K] that sum in 2^-40 units << 16 | parts added
-    long long* trace;
     int T, slice_vecs;
 };
 
@@ -107,12 +108,10 @@ __device__ __forceinline__ bool spin_ge(const int* p, int want) {
 // fp32-summed normalisers.  Measured on 40 000 draws with the certification switched off, the largest
 // error that changed a token was 0.1 * delta * sqrt(sum p^2 + q^2); kappa = 4 leaves a factor 40 over
 // that.
-#ifndef BEBOP_KAPPA
-#define BEBOP_KAPPA 4.0
-#endif
-__device__ __forceinline__ double draw_bound(double sumsq) {
+constexpr double kDrawKappa = 4.0;
+__device__ __forceinline__ double draw_bound(double sumsq, double kappa = kDrawKappa) {
     const double delta = 2.384185791015625e-07;   // 2^-22
-    return BEBOP_KAPPA * delta * sqrt(sumsq) + 1e-300;
+    return kappa * delta * sqrt(sumsq) + 1e-300;
 }
 
 // c = log2(e) / tau in fp32, and 2^(x * c - E): the product is exact inside the fma, so the argument
@@ -134,11 +133,11 @@ __device__ __forceinline__ int ref_exponent(float m, const TempScale& t, float* 
     return ceil_alu(th, Ef);
 }
 
-struct WaveShared {
+struct DrawShared {
     double redd[WW];
     float redf[2][WW];
     int redi[WW];
-    int ticket, phase, wave, index;
+    int ticket, phase, index;
     // D-phase broadcast
     double base, Ttarget, bound;
     int owner_slice;

@@ -1,27 +1,8 @@
 // The fp64 re-draw of the sequences whose fast draw did not clear its error bound (its first kernel also turns
-// an expired device-side wait into a status bit), and the hooks that time and trace the main kernel.
+// an expired device-side wait into a status bit), and the hook that times the main kernel.
 #include "bebop_pipe.cuh"
 
 namespace bebop {
-
-#ifdef BEBOP_TRACE
-// timeline of the re-draw kernel: [2i] earliest, [2i+1] latest global-timer stamp of event i over all CTAs
-__device__ unsigned long long g_redraw_trace[32];
-__device__ __forceinline__ void xt_log(int i) {
-    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    atomicMin(&g_redraw_trace[2 * i], t); atomicMax(&g_redraw_trace[2 * i + 1], t);
-}
-#define XTLOG(i) do { if (threadIdx.x == 0) xt_log(i); } while (0)
-extern "C" void bebop_debug_redraw_trace(unsigned long long* host32, int reset) {
-    if (reset) {
-        unsigned long long init[32];
-        for (int i = 0; i < 16; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
-        cudaMemcpyToSymbol(g_redraw_trace, init, sizeof(init));
-    } else cudaMemcpyFromSymbol(host32, g_redraw_trace, 32 * sizeof(unsigned long long));
-}
-#else
-#define XTLOG(i) do { } while (0)
-#endif
 
 namespace {
 
@@ -53,6 +34,7 @@ struct RedrawArgs {
     double* xmass;           // [B][XT][WW] residual mass per quarter slice and warp chunk
     int* xsdone;             // [B] per listed sequence: sum tasks finished
     int* xdone;              // [B] per listed sequence: mass tasks finished
+    int expire;              // test hook: the wait for the list gives up at once
     unsigned* xticket;       // [1] next work item
     int T, slice_vecs;
 };
@@ -61,9 +43,6 @@ struct RedrawArgs {
 // 2^f by its series to the fifth power (the next term is below 4e-17 of the result).  About a dozen
 // double-precision instructions, a third of the library routine; the result is within 2 ulp.
 // `tab` holds 2^(j/64), j = 0..63, in shared memory.  Arguments below -1000 (and -inf) give 0.
-#ifndef BEBOP_XPOLL
-#define BEBOP_XPOLL 256
-#endif
 constexpr int XTAB = 64;
 __device__ __forceinline__ void x_exp2_table(double* tab) {
     if (threadIdx.x < XTAB) tab[threadIdx.x] = exp2((double)threadIdx.x * (1.0 / XTAB));
@@ -167,12 +146,13 @@ __device__ __forceinline__ unsigned long long x_ld_count(const unsigned long lon
 }
 // 1: slot is listed and its record is valid; 0: the list is complete and ends before it; -1: a wait gave up
 __device__ __forceinline__ int x_wait_slot(const RedrawArgs& a, int slot) {
+    if (a.expire) return -1;                             // test hook: this wait's bound has run out already
     uint32_t i = 0;
     for (; i < kSpin; ++i) {
         const unsigned long long w = x_ld_count(a.fb_count);
         if (slot < (int)(w & 0xffffffffull)) break;
         if ((int)(w >> 32) >= a.expect) return 0;
-        __nanosleep(BEBOP_XPOLL);
+        __nanosleep(256);
     }
     if (i == kSpin) return -1;
     for (i = 0; i < kSpin; ++i) {                       // a place in the list is taken before its record is written
@@ -215,7 +195,6 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             if (g < 0 && tid == 0) atomicExch(a.wait_failed, 1);
             break;
         }
-        XTLOG(0);
         XRow d;
         x_row(a, slot, &d);
         const int b = d.b;
@@ -242,7 +221,6 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             sa = warp_sum(sa); sb = warp_sum(sb);
             if (lane == 0) { sh[0][warp] = sa; sh[1][warp] = sb; }
             __syncthreads();
-            XTLOG(1);
             if (tid == 0) {
                 double ta = 0.0, tb = 0.0;
                 for (int w = 0; w < WW; ++w) { ta += sh[0][w]; tb += sh[1][w]; }
@@ -262,7 +240,6 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
         }
         // exact normalisers: every warp adds the quarter-slice sums in the same order (lane t takes sums t,
         // t + 32, ...; the butterfly leaves the same bits in every lane), so every CTA gets the same value
-        XTLOG(3);
         double Sa = 0.0, Sb = 0.0;
         for (int t = lane; t < XT; t += 32) { const double2 x = __ldcg(a.xsum + (int64_t)b * XT + t); Sa += x.x; Sb += x.y; }
         Sa = warp_sum(Sa); Sb = warp_sum(Sb);
@@ -286,7 +263,6 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             S.last = atomicAdd(a.xdone + slot, 1) == XT - 1;
         }
         __syncthreads();
-        XTLOG(4);
         if (!S.last) continue;
         __threadfence();
 
@@ -324,7 +300,6 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
             S.target = t; S.base = C;
         }
         __syncthreads();
-        XTLOG(5);
         const int qs = S.sel;
         // Stage 2: warp chunk inside the quarter slice (residual: stored; plain softmax row: evaluated now)
         const int p0 = qs * qv, pn = max(min(qv, R.nvec - p0), 0);
@@ -392,23 +367,21 @@ __global__ void __launch_bounds__(WT) k_redraw(const RedrawArgs a) {
         if (lastpos >= 0) atomicMax(&S.tok_last, lastpos);
         __syncthreads();
         if (tid == 0) a.o.out_tokens[(int64_t)b * (K + 1) + d.k] = S.tok_first != 0x7fffffff ? S.tok_first : S.tok_last;
-        XTLOG(7);
         __syncthreads();
     }
+    // Every CTA waits here for the main grid, whatever the caller asked for: a dependent of a grid that lets its
+    // dependents start early has to, or work enqueued behind this kernel (a copy of the results, the next call's
+    // clearing of this workspace) would not be ordered behind that grid.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // a wait that gave up, in the main kernel or here: every row's status says so
-    if (a.o.row_status) {
-        asm volatile("griddepcontrol.wait;" ::: "memory");       // the main grid is through and its writes are visible
-        if (ld_acquire(a.wait_failed) != 0)
-            for (int b = blockIdx.x * WT + tid; b < R.B; b += gridDim.x * WT) atomicOr(a.o.row_status + b, ST_WAIT);
-    }
+    if (a.o.row_status && ld_acquire(a.wait_failed) != 0)
+        for (int b = blockIdx.x * WT + tid; b < R.B; b += gridDim.x * WT) atomicOr(a.o.row_status + b, ST_WAIT);
 }
 
 }  // namespace
 
-long long* g_wave_trace = nullptr;
-void wave_set_trace(long long* p) { g_wave_trace = p; }
 cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
-void wave_set_events(cudaEvent_t start, cudaEvent_t stop) { g_ev_start = start; g_ev_stop = stop; }
+void pipe_set_events(cudaEvent_t start, cudaEvent_t stop) { g_ev_start = start; g_ev_stop = stop; }
 
 namespace {
 template <int DT>
@@ -437,8 +410,9 @@ int redraw_grid() {
 // `expect` sequences get their draw decided by the main kernel (0: none, nothing is listed).
 cudaError_t redraw_launch(const RowArgs& a, const float* u_final, VerifyOut o, const unsigned long long* fb_count,
                           const FbRec* fb_list, int expect, int* wait_failed, char* w,
-                          const WavePlan& wp, cudaStream_t stream) {
+                          const PipePlan& wp, cudaStream_t stream, bool expire_list_wait) {
     RedrawArgs ra;
+    ra.expire = expire_list_wait ? 1 : 0;
     ra.r = a; ra.u_final = u_final; ra.o = o;
     ra.fb_count = fb_count; ra.fb_list = fb_list; ra.expect = expect;
     ra.wait_failed = wait_failed;

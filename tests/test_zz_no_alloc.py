@@ -39,6 +39,36 @@ def test_static_equals_workspace_two_calls_in_a_row(dtype, N, V):
             assert float(got["tv"][2]) == 0.0 and int(got["row_status"][3]) & 1
 
 
+def test_static_against_the_oracle():
+    """One small comparison with the fp64 oracle, so that this entry point does not stand on bebop_tv alone."""
+    import numpy as np
+    import oracle
+    import paper_2606_12370_b200 as P
+    tgt, drf, tau = _inputs(7, 12, 4100, torch.float32)
+    got = P.bebop_tv_static(tgt, drf, temperature=tau)
+    ref = oracle.tv(tgt.cpu().numpy(), drf.cpu().numpy(), temperature=tau.cpu().numpy())
+    assert np.abs(got["tv"].cpu().numpy() - ref["tv"]).max() <= 1e-5
+    assert np.abs(got["s_aux"].cpu().numpy() - ref["s_aux"]).max() <= 1e-5
+    assert (got["row_status"].cpu().numpy() == ref["row_status"]).all()
+
+
+def test_static_limit_is_where_the_header_says():
+    """The largest shape the built-in scratch takes (rows in one slice: 24 bytes per row pair in two 256-byte aligned
+    arrays of one MiB together, i.e. 43,680 row pairs) runs and equals bebop_tv; one row pair more is refused."""
+    import paper_2606_12370_b200 as P
+    N, V = 43680, 8
+    tgt, drf, tau = _inputs(9, N + 1, V, torch.bfloat16)
+    got = P.bebop_tv_static(tgt[:N], drf[:N], temperature=tau[:N])
+    P.bebop_debug_force_general_path(1)
+    want = P.bebop_tv(tgt[:N], drf[:N], temperature=tau[:N])
+    P.bebop_debug_force_general_path(0)
+    torch.cuda.synchronize()
+    assert torch.equal(got["tv"].view(torch.int32), want["tv"].view(torch.int32))
+    with pytest.raises(P.BebopError) as e:
+        P.bebop_tv_static(tgt, drf, temperature=tau)
+    assert e.value.code == 9
+
+
 def test_static_rejects_what_does_not_fit():
     import paper_2606_12370_b200 as P
     N, V = 50000, 1024                           # 50,000 row pairs x 1 slice x 24 B > 1 MiB
