@@ -21,10 +21,11 @@
 // eight partials, hands the stage back, merges them in warp order and publishes.  No CTA-wide barrier
 // sits on the streaming path.
 //
-// What CTAs pass to each other through global memory needs no fence: 16-byte records written by one
-// store and carrying a validity mark (the memory starts at zero), and fixed-point sums with a count of
-// contributions in the low bits of the same word, added by relaxed atomics.  Counters only say when to
-// look; whoever looks checks the marks and waits (bounded) for a record that is not there yet.
+// What CTAs pass to each other through global memory needs no fence: records of two 64-bit words, both
+// non-zero once written (the memory starts at zero), which a reader takes only when it sees both; and
+// fixed-point sums with a count of contributions in the low bits of the same word, added by relaxed atomics.
+// Counters only say when to look; whoever looks checks the record and waits (bounded) for one that is not
+// there yet.
 //
 // Every wait is bounded; a wait that gives up sets the wait flag (status bit 32 of every row).
 // No multicast, no cluster: each CTA copies from this GPU's own memory.
@@ -208,9 +209,9 @@ __device__ __forceinline__ void producer(const PipeArgs& a, PipeShared& S, unsig
     // waited for only when the shelf is full or no tickets are left.
     // the sequence's record of the accept scan, valid once its mark is set (waits, bounded, if asked to)
     auto seq_info = [&](int b, bool wait) {
-        SeqInfo si = ld_cg(a.sinfo + b);
+        SeqInfo si = ld_seq(a.sinfo + b);
         if (a.expire) { if (wait) si.pad = 0; return si; }          // test hook: this wait's bound has run out already
-        if (wait) for (uint32_t i = 0; si.pad == 0 && i < kSpin; ++i) { __nanosleep(64); si = ld_cg(a.sinfo + b); }
+        if (wait) for (uint32_t i = 0; si.pad == 0 && i < kSpin; ++i) { __nanosleep(64); si = ld_seq(a.sinfo + b); }
         return si;
     };
     SeqInfo seen; seen.n = 0; seen.draw_row = 0; seen.pad0 = 0; seen.pad = 0;     // the record `ready` last saw valid,
@@ -322,7 +323,7 @@ __device__ __forceinline__ void producer(const PipeArgs& a, PipeShared& S, unsig
                 row0 = row_ptr(R, b, r);
             } else {
                 // everything the row needs is requested at once (the sequence was seen ready: its records are there)
-                const SeqInfo si = seen_b == b ? seen : ld_cg(a.sinfo + b);
+                const SeqInfo si = seen_b == b ? seen : ld_seq(a.sinfo + b);
                 // row 0 of the sequence's second sweep is the row its token is drawn from; the others follow in order
                 const bool drawrow = !TVO && r == 0;
                 const int rp = TVO ? r : r - 1;
@@ -334,8 +335,8 @@ __device__ __forceinline__ void producer(const PipeArgs& a, PipeShared& S, unsig
                 // (the accept scan saw these row records before it set the sequence's mark; should a load have
                 // overtaken that all the same, ask again)
                 const bool no_row_k = TVO && k >= L;      // bebop_tv has no bonus row: nothing was merged for it
-                if (k <= L && !no_row_k) for (uint32_t i = 0; !(sp.st & kRowValid) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
-                if (k < L) for (uint32_t i = 0; !(sq.st & kRowValid) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
+                if (k <= L && !no_row_k) for (uint32_t i = 0; !rec_valid(sp) && i < kSpin; ++i) sp = ld_cg(a.rstat + (int64_t)b * NR + k);
+                if (k < L) for (uint32_t i = 0; !rec_valid(sq) && i < kSpin; ++i) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k);
                 d.c = __int_as_float(si.pad0);
                 const bool pair = k < L;
                 skip = k > L || si.n < 0 || (!pair && !(drawrow && si.draw_row == L)) || no_row_k;
@@ -366,6 +367,14 @@ __device__ __forceinline__ void producer(const PipeArgs& a, PipeShared& S, unsig
     }
 }
 
+// a merged row's record (it has been seen by the sequence's accept scan; should this thread's load run ahead of that
+// all the same, it asks again)
+__device__ __forceinline__ RowStat ld_row(const PipeArgs& a, int64_t i) {
+    RowStat x = ld_cg(a.rstat + i);
+    for (uint32_t k = 0; !rec_valid(x) && k < kSpin; ++k) { __nanosleep(64); x = ld_cg(a.rstat + i); }
+    return x;
+}
+
 // ------------------------------------------------------------------ phase A without tickets
 // The warp that delivers the last softmax partial of a ROW merges that row's partials (exactly:
 // integer exponents, fp64 sums in a fixed tree) and leaves the row's normaliser; the warp that merges
@@ -381,10 +390,10 @@ __device__ __forceinline__ void merge_row_warp(const PipeArgs& a, int b, int r) 
     P1Part mine[2];
     int cnt = 0;
     for (int s = lane; s < T && cnt < 2; s += 32) {
-        // the record's exponent is stored as 2e + 1: zero means the record is not there yet
+        // (the record's exponent is stored as 2e + 1, its sum with non-zero bits: a record is there when both words are)
         P1Part rec = ld_cg(pp + s);
-        for (uint32_t i = 0; rec.e == 0 && i < kSpin; ++i) { __nanosleep(64); rec = ld_cg(pp + s); }
-        if (rec.e == 0) atomicExch(a.wait_failed, 1);
+        for (uint32_t i = 0; !rec_valid(rec) && i < kSpin; ++i) { __nanosleep(64); rec = ld_cg(pp + s); }
+        if (!rec_valid(rec)) { atomicExch(a.wait_failed, 1); rec.e = 2 * E_EMPTY + 1; rec.s = 0.0; rec.m = 0.f; }
         rec.e = (rec.e - 1) >> 1;
         mine[cnt] = rec; e_l = max(e_l, rec.e);
         if (rec.m != rec.m) f_l = 1;
@@ -397,7 +406,7 @@ __device__ __forceinline__ void merge_row_warp(const PipeArgs& a, int b, int r) 
     if (lane == 0) {
         int st = 0;
         if (f_l || !(s_l == s_l)) st = ST_NONFINITE; else if (Em == E_EMPTY) st = ST_EMPTY;
-        RowStat rs; rs.inv_s = (!st && s_l > 0.0) ? 1.0 / s_l : 0.0; rs.e = Em; rs.st = st | kRowValid;
+        RowStat rs; rs.inv_s = nonzero_bits((!st && s_l > 0.0) ? 1.0 / s_l : 0.0); rs.e = Em; rs.st = st | kRowValid;
         st16(a.rstat + (int64_t)b * NR + r, rs);
     }
 }
@@ -420,8 +429,8 @@ __device__ __noinline__ void accept_warp(const PipeArgs& a, int b) {
     sq = sp;
     auto row = [&](int r) {                                            // a merged row's record (waits, bounded, for its mark)
         RowStat x = ld_cg(a.rstat + (int64_t)b * NR + r);
-        for (uint32_t i = 0; x.st == 0 && i < kSpin; ++i) { __nanosleep(64); x = ld_cg(a.rstat + (int64_t)b * NR + r); }
-        if (x.st == 0) atomicExch(a.wait_failed, 1);
+        for (uint32_t i = 0; !rec_valid(x) && i < kSpin; ++i) { __nanosleep(64); x = ld_cg(a.rstat + (int64_t)b * NR + r); }
+        if (!rec_valid(x)) { atomicExch(a.wait_failed, 1); x.inv_s = 0.0; x.e = E_EMPTY; x.st = ST_WAIT; }
         x.st &= 0xff;
         return x;
     };
@@ -467,7 +476,7 @@ __device__ __noinline__ void accept_warp(const PipeArgs& a, int b) {
         // the record's mark makes it (and, through the row records it was computed from, the sequence) ready
         // (pad0 carries c = log2(e) / tau of the sequence: the second sweep's producer need not divide again)
         SeqInfo si; si.n = fatal ? -1 : nn; si.draw_row = (fatal || tvo) ? -1 : nn; si.pad0 = __float_as_int(ts.hi); si.pad = 1;
-        st16(a.sinfo + b, si);
+        st_seq(a.sinfo + b, si);
         if (fatal && !tvo) draw_decided(a.fb_count);     // no draw will come
     }
 }
@@ -704,14 +713,14 @@ __device__ __noinline__ void draw_setup_warp(const PipeArgs& a, PipeShared& S, i
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, NR = 2 * K + 1, L = len_of(R, b), T2 = 2 * a.T;
-    const SeqInfo si = ld_cg(a.sinfo + b);
+    const SeqInfo si = ld_seq(a.sinfo + b);
     if (si.n < 0) return;
     const int k = si.draw_row;
     const bool pair = k >= 0 && k < L;
     // lane 0 will need the draw rows' records: asked for now, with everything else
     RowStat sp, sq;
     sp.inv_s = 0.0; sp.e = 0; sp.st = 0; sq = sp;
-    if (lane == 0 && k >= 0 && (what & 2)) { sp = ld_cg(a.rstat + (int64_t)b * NR + k); if (pair) sq = ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k); }
+    if (lane == 0 && k >= 0 && (what & 2)) { sp = ld_row(a, (int64_t)b * NR + k); if (pair) sq = ld_row(a, (int64_t)b * NR + K + 1 + k); }
     if ((what & 1) && lane < L && a.o.tv) {
         // the position's TV parts were added in fixed point, with a count of one each in the low 16 bits
         unsigned long long w = 0;
@@ -751,9 +760,7 @@ __device__ __noinline__ void draw_setup_warp(const PipeArgs& a, PipeShared& S, i
         if (!(Tt > 0.0)) owner = -1;
         if (owner < 0) {
             // no half slice owns the target (no residual mass, or u = 0): the fp64 re-draw decides
-            FbRec rec;
-            rec.b1 = b + 1; rec.kp = 2 * k + (pair ? 1 : 0); rec.ep = sp.e; rec.eq = pair ? sq.e : 0;
-            st16(a.fb_list + draw_listed(a.fb_count), rec);
+            st_fb(a.fb_list + draw_listed(a.fb_count), b, 2 * k + (pair ? 1 : 0), sp.e, pair ? sq.e : 0);
         } else {
             // the mailbox has room for more draws than this CTA's unpublished tasks can bring; should it be full
             // all the same, wait (bounded) for the producer
@@ -866,11 +873,8 @@ __device__ __forceinline__ void pipe_d(const PipeArgs& a, PipeShared& PS, const 
         for (int w = 0; w < WW; ++w) if (S.redi[w] != -1) { y = S.redi[w]; cnt++; }
         if (cnt == 1 && y >= 0) { a.o.out_tokens[(int64_t)b * (K + 1) + k] = y; draw_decided(a.fb_count); }
         else {
-            FbRec rec;
-            rec.b1 = b + 1; rec.kp = 2 * k + (pair ? 1 : 0);
-            rec.ep = ld_cg(a.rstat + (int64_t)b * NR + k).e;
-            rec.eq = pair ? ld_cg(a.rstat + (int64_t)b * NR + K + 1 + k).e : 0;
-            st16(a.fb_list + draw_listed(a.fb_count), rec);
+            st_fb(a.fb_list + draw_listed(a.fb_count), b, 2 * k + (pair ? 1 : 0), ld_row(a, (int64_t)b * NR + k).e,
+                  pair ? ld_row(a, (int64_t)b * NR + K + 1 + k).e : 0);
         }
     }
 }
@@ -921,7 +925,7 @@ __device__ __forceinline__ void publisher(const PipeArgs& a, PipeShared& S) {
 #pragma unroll
             for (int o = 4; o > 0; o >>= 1) im = min(im, __shfl_xor_sync(0xffffffffu, im, o));
             if (lane == 0) {
-                P1Part p; p.s = (double)im; p.e = 1; p.m = ord2f(om);
+                P1Part p; p.s = nonzero_bits((double)im); p.e = 1; p.m = ord2f(om);
                 st16(a.part + ((int64_t)b * (2 * K + 1) + r) * a.T + sl, p);
             }
         } else if (phase == 0) {
@@ -937,8 +941,8 @@ __device__ __forceinline__ void publisher(const PipeArgs& a, PipeShared& S) {
             int run_a = 0;
             if (lane == 0) {
                 // the slice's record (exponent stored as 2e + 1: zero means "not there yet"), then the row's counter.
-                // No fence: whoever the counter wakes checks every record's mark before using it.
-                P1Part p; p.s = (mc != mc) ? 0.0 : sum; p.e = 2 * Ec + 1; p.m = mc;
+                // No fence: whoever the counter wakes checks that both words of every record are there before using it.
+                P1Part p; p.s = nonzero_bits((mc != mc) ? 0.0 : sum); p.e = 2 * Ec + 1; p.m = mc;
                 st16(a.part + ((int64_t)b * (2 * K + 1) + r) * a.T + sl, p);
                 run_a = atomicAdd(&a.rowcnt[(int64_t)b * (2 * K + 1) + r], 1) == a.T - 1;
             }

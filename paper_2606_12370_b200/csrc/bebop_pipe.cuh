@@ -19,13 +19,28 @@ constexpr uint32_t kSpin = 1u << 22;
 struct __align__(16) P1Part { double s; int e; float m; };             // per (row, slice); m = NaN marks a non-finite logit
 struct __align__(16) RowStat { double inv_s; int e; int st; };   // per row, after the merge: 1/S, exponent E, status bits | kRowValid
 constexpr int kRowValid = 0x100;
-// One 16-byte store of a 16-byte record: a reader that sees the record's validity mark sees all of it.  The
-// records that CTAs pass to each other start at zero and carry such a mark, so they need no fence.
-template <typename T> __device__ __forceinline__ void st16(T* p, const T& v) {
+// Records that CTAs pass to each other through global memory (the memory starts at zero).  A record is two
+// 8-byte words, written by one store of two 64-bit elements and read by one such load.  The PTX memory model
+// treats a vector access as its elements accessed in no particular order, each 64-bit element being a single
+// copy; so every record is laid out with BOTH words non-zero once written (a zero sum is stored as -0.0, counts
+// and exponents carry an offset or a low mark bit), and a reader takes a record only when both words are
+// non-zero: each word then is the written one.  No fence is needed for that, and none is used.
+template <typename T> __device__ __forceinline__ void rec_words(const T& v, unsigned long long* w) {
     static_assert(sizeof(T) == 16, "16-byte record");
-    const uint4 b = *reinterpret_cast<const uint4*>(&v);
-    asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" :: "l"(p), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+    memcpy(w, &v, 16);
 }
+template <typename T> __device__ __forceinline__ void st16(T* p, const T& v) {
+    unsigned long long w[2];
+    rec_words(v, w);
+    asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" :: "l"(p), "l"(w[0]), "l"(w[1]) : "memory");
+}
+template <typename T> __device__ __forceinline__ bool rec_valid(const T& v) {
+    unsigned long long w[2];
+    rec_words(v, w);
+    return w[0] != 0ull && w[1] != 0ull;
+}
+// a sum that may be exactly zero, made non-zero in its bits
+__device__ __forceinline__ double nonzero_bits(double x) { return x == 0.0 ? -0.0 : x; }
 struct __align__(16) DPart { double tot; float sq; int pad; };        // per (sequence, slice)
 struct __align__(16) SeqInfo {          // per sequence, written by phase A
     int n;                              // accept count (stop position); -1: fatal
@@ -82,14 +97,36 @@ __device__ __forceinline__ void draw_decided(unsigned long long* w) {
 __device__ __forceinline__ int draw_listed(unsigned long long* w) {
     return (int)(atomicAdd(w, (1ull << 32) | 1ull) & 0xffffffffull);
 }
-// Workspace records written by other CTAs of this launch are read through L2 only: the L1 of this SM
-// may hold an older copy of the line (a neighbouring record read earlier).
+// Workspace records written by other CTAs of this launch: one load of two 64-bit elements, at GPU scope (the L1 of
+// this SM may hold an older copy of the line).  Use the record only if rec_valid() says both words are there.
 template <typename T> __device__ __forceinline__ T ld_cg(const T* p) {
-    static_assert(sizeof(T) % 16 == 0, "16-byte records");
+    static_assert(sizeof(T) == 16, "16-byte record");
+    unsigned long long w[2];
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w[0]), "=l"(w[1]) : "l"(p) : "memory");
     T r;
-#pragma unroll
-    for (int i = 0; i < (int)(sizeof(T) / 16); ++i)
-        reinterpret_cast<uint4*>(&r)[i] = __ldcg(reinterpret_cast<const uint4*>(p) + i);
+    memcpy(&r, w, 16);
+    return r;
+}
+// SeqInfo in memory: n and draw_row (both >= -1) are stored plus 2 and pad as 1, so that both words are non-zero (pad0 is
+// the bit pattern of a positive float).  In registers the fields are plain again and pad says whether the record was there.
+__device__ __forceinline__ void st_seq(SeqInfo* p, const SeqInfo& s) {
+    SeqInfo m; m.n = s.n + 2; m.draw_row = s.draw_row + 2; m.pad0 = s.pad0; m.pad = 1;
+    st16(p, m);
+}
+__device__ __forceinline__ SeqInfo ld_seq(const SeqInfo* p) {
+    const SeqInfo m = ld_cg(p);
+    SeqInfo s; s.n = m.n - 2; s.draw_row = m.draw_row - 2; s.pad0 = m.pad0; s.pad = rec_valid(m) ? 1 : 0;
+    return s;
+}
+// FbRec in memory: the exponents as 2 e + 1 (b1 = sequence + 1 is non-zero already)
+__device__ __forceinline__ void st_fb(FbRec* p, int b, int kp, int ep, int eq) {
+    FbRec r; r.b1 = b + 1; r.kp = kp; r.ep = 2 * ep + 1; r.eq = 2 * eq + 1;
+    st16(p, r);
+}
+__device__ __forceinline__ FbRec ld_fb(const FbRec* p, bool* valid) {
+    const FbRec m = ld_cg(p);
+    *valid = rec_valid(m);
+    FbRec r; r.b1 = m.b1; r.kp = m.kp; r.ep = m.ep >> 1; r.eq = m.eq >> 1;      // (2 e + 1) >> 1 = e, for negative e too
     return r;
 }
 __device__ __forceinline__ bool spin_ge(const int* p, int want) {

@@ -78,7 +78,8 @@ __device__ __forceinline__ double x_resid(const XRow& d, float zp, float zq, con
 }
 __device__ __forceinline__ void x_row(const RedrawArgs& a, int slot, XRow* d) {
     const RowArgs& R = a.r;
-    const FbRec rec = ld_cg(a.fb_list + slot);
+    bool there;
+    const FbRec rec = ld_fb(a.fb_list + slot, &there);          // (x_wait_slot has seen the record valid)
     const int b = rec.b1 - 1, k = rec.kp >> 1;
     d->b = b; d->k = k;
     d->pair = rec.kp & 1;
@@ -156,7 +157,7 @@ __device__ __forceinline__ int x_wait_slot(const RedrawArgs& a, int slot) {
     }
     if (i == kSpin) return -1;
     for (i = 0; i < kSpin; ++i) {                       // a place in the list is taken before its record is written
-        if (ld_cg(a.fb_list + slot).b1 != 0) return 1;
+        if (rec_valid(ld_cg(a.fb_list + slot))) return 1;
         __nanosleep(64);
     }
     return -1;
