@@ -83,6 +83,54 @@ def _worker(rank, world, port, ret):
         dist.destroy_process_group()
 
 
+def _bench_worker(rank, world, port, ret):
+    """Two ranks go through bench.py's own per-rank function (strong scaling over a small ragged batch); the oracle
+    stands in for the device step."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import bench
+        import oracle
+        over = {"B": 13, "V": 640}
+        wl = bench.rank_workload(rank, world, "strong", "cpu", over)
+        x, cfg = wl["x"], wl["cfg"]
+        res = oracle.verify(x["target"].float().numpy(), x["draft"].float().numpy(), x["draft_tokens"].numpy(),
+                            x["u_accept"].numpy(), x["u_final"].numpy(), draft_len=x["draft_len"].numpy(),
+                            temperature=x["temperature"].numpy(), nthreads=1)
+        mine = torch.full((cfg.B, cfg.K + 2), -9, dtype=torch.int64)
+        sl = slice(wl["begin"], wl["end"])
+        mine[sl, 0] = torch.from_numpy(res["accept_len"].astype(np.int64))
+        mine[sl, 1:] = torch.from_numpy(res["out_tokens"].astype(np.int64))
+        dist.all_reduce(mine, op=dist.ReduceOp.MAX)
+        tot = torch.tensor([wl["positions"], wl["rows"], wl["nseq"]], dtype=torch.float64)
+        dist.all_reduce(tot)
+        edges = torch.zeros(world, 2, dtype=torch.int64)
+        edges[rank, 0], edges[rank, 1] = wl["begin"], wl["end"]
+        dist.all_reduce(edges)
+        if rank == 0:
+            whole = bench.rank_workload(0, 1, "strong", "cpu", over)
+            xf = whole["x"]
+            full = oracle.verify(xf["target"].float().numpy(), xf["draft"].float().numpy(), xf["draft_tokens"].numpy(),
+                                 xf["u_accept"].numpy(), xf["u_final"].numpy(), draft_len=xf["draft_len"].numpy(),
+                                 temperature=xf["temperature"].numpy(), nthreads=1)
+            ret["same"] = bool((mine[:, 0].numpy() == full["accept_len"]).all() and (mine[:, 1:].numpy() == full["out_tokens"]).all())
+            ret["totals"] = [float(v) for v in tot] == [float(whole["positions"]), float(whole["rows"]), float(whole["nseq"])]
+            ret["cover"] = edges[0, 0].item() == 0 and edges[-1, 1].item() == cfg.B and all(
+                edges[r, 1].item() == edges[r + 1, 0].item() for r in range(world - 1))
+            rows = [int((2 * xf["draft_len"][edges[r, 0]:edges[r, 1]].long() + 1).sum()) for r in range(world)]
+            ret["balanced"] = max(rows) - min(rows) <= 2 * (2 * cfg.K + 1)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_bench_rank_function_strong_scaling_two_ranks():
+    mgr = mp.Manager()
+    ret = mgr.dict()
+    mp.spawn(_bench_worker, args=(2, _free_port(), ret), nprocs=2, join=True)
+    assert ret["same"] and ret["totals"] and ret["cover"] and ret["balanced"], dict(ret)
+
+
 def test_two_ranks_equal_one():
     mgr = mp.Manager()
     ret = mgr.dict()
