@@ -162,16 +162,19 @@ bebop_status_t bebop_greedy_verify(
 /*
  * Test and measurement hooks (no counterpart in the paper).  They set process-wide switches that every later
  * call in the process sees: not thread-safe, and not meant for code that serves requests.
- * bebop_debug_force_general_path(1) makes bebop_verify, bebop_tv and bebop_greedy_verify use the
- * split-row general kernels even for shapes the pipelined kernel takes (0 restores the default).
+ * bebop_debug_force_general_path(mode) chooses the kernels behind bebop_verify, bebop_tv and bebop_greedy_verify:
+ * 0 (the default) the faster, by measurement, of the fused and the pipelined kernel for the shape, and the
+ * split-row general kernels for shapes neither takes; 1 the general kernels always; 2 never the fused kernel;
+ * 3 the fused kernel wherever it applies (the greedy mode has no fused form).  All give the same results up to
+ * the documented tolerances.
  * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
  * shape, of an int32 that after a bebop_verify call holds the number of sequences
  * whose draw was re-done by the fp64 kernels.
  * bebop_debug_set_timing_events(start, stop): two cudaEvent_t handles that the next
- * bebop_verify calls record around the pipelined kernel, on the caller's stream (NULL,
+ * bebop_verify calls record around the main (pipelined or fused) kernel, on the caller's stream (NULL,
  * NULL switches it off).
  * bebop_debug_expire_wait(which): the next call's device-side wait number `which` (1: the re-draw kernel's wait
- * for the list of sequences; 2: the pipelined kernel's wait for a sequence's accept scan) gives up at once, as if
+ * for the list of sequences; 2: the main kernel's wait for what other CTAs deliver) gives up at once, as if
  * its bound had run out: the call still returns, every row_status carries BEBOP_ROW_WAIT_EXPIRED, and the call
  * after it is normal again (0: off).  For the test of the bounded waits; nothing is trapped or hung.
  * bebop_debug_set_draw_kappa(kappa): the factor in the error bound that decides whether bebop_verify keeps a token

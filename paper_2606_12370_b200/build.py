@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbebop.so")
-SOURCES = ["bebop_api.cu", "bebop_general.cu", "bebop_redraw.cu", "bebop_pipe.cu"]
+SOURCES = ["bebop_api.cu", "bebop_general.cu", "bebop_redraw.cu", "bebop_pipe.cu", "bebop_fuse.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-shared"]

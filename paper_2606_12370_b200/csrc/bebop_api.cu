@@ -9,7 +9,8 @@ namespace {
 
 // Test hook: route bebop_verify through the general (split-row) path even where the fused
 // kernel applies, so that both paths are covered by the parity tests.
-int g_path = 0;   // 0: pipelined kernel where it applies, else the general kernels; 1: general kernels only
+int g_path = 0;   // 0: the faster of the fused and the pipelined kernel where they apply, else the general kernels;
+                  // 1: general kernels only; 2: never the fused kernel; 3: the fused kernel wherever it applies
 
 int g_expire_wait = 0;   // test hook: which device-side wait the next call lets give up at once
 float g_draw_kappa = -1.f;   // test hook: factor of the fast draw's error bound (negative: the built-in value)
@@ -110,7 +111,9 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 0 && pipe_supported(a))
+    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, false))) && fuse_supported(a))
+        e = fuse_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
+    if (e == cudaSuccess && !launched && g_path != 1 && pipe_supported(a))
         e = pipe_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
     if (e == cudaSuccess && !launched) e = general_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
@@ -135,9 +138,11 @@ bebop_status_t bebop_tv(const void* target_logits, int64_t ld_target, const void
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 0 && pipe_supported(a)) {
+    VerifyOut o{nullptr, nullptr, tv, nullptr, nullptr, row_status};
+    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, true))) && fuse_supported(a))
+        e = fuse_verify(a, p, nullptr, nullptr, nullptr, o, static_cast<char*>(workspace), stream, &launched, true, s_aux);
+    if (e == cudaSuccess && !launched && g_path != 1 && pipe_supported(a)) {
         // the pipelined kernel with row pairs in place of sequences: first sweep, second sweep, no draw
-        VerifyOut o{nullptr, nullptr, tv, nullptr, nullptr, row_status};
         e = pipe_verify(a, p, nullptr, nullptr, nullptr, o, static_cast<char*>(workspace), stream, &launched, true, s_aux);
     }
     if (e == cudaSuccess && !launched)
@@ -163,7 +168,7 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path == 0 && pipe_supported(a))
+    if (g_path != 1 && pipe_supported(a))
         e = pipe_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream, &launched);
     if (e == cudaSuccess && !launched)
         e = general_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream);

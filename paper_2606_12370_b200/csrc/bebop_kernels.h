@@ -64,6 +64,15 @@ cudaError_t pipe_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
                         const float* u_accept, const float* u_final, VerifyOut o, char* ws,
                         cudaStream_t stream, bool* launched, bool tv_only = false, float* s_aux = nullptr);
 
+// Fused kernel (bebop_fuse.cu): every row read and exponentiated once, the exponentials parked in tensor memory
+// between the softmax statistics and the residuals; same contract as pipe_verify.  fuse_preferred says whether,
+// by measurement, it is the faster of the two for the shape.
+bool fuse_supported(const RowArgs& a);
+bool fuse_preferred(const RowArgs& a, bool tv_only);
+cudaError_t fuse_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens,
+                        const float* u_accept, const float* u_final, VerifyOut o, char* ws,
+                        cudaStream_t stream, bool* launched, bool tv_only = false, float* s_aux = nullptr);
+
 // The greedy mode through the pipelined kernel: one sweep over the target rows (maximum and lowest index per
 // slice), then a small kernel that merges the slices and runs the argmax match.
 cudaError_t pipe_greedy(const RowArgs& a, const Plan& p, const int32_t* draft_tokens, int32_t* accept_len,

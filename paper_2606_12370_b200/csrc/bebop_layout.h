@@ -40,7 +40,28 @@ struct Plan {
     size_t off_dmass;   // double [B][nsplit_d]          residual / bonus mass partials
     size_t off_amax;    // float,int [B][K+1][nsplit]    argmax partials (greedy)
     size_t off_pipe;    // workspace of the pipelined kernel
+    size_t off_fuse;    // workspace of the fused kernel (the same bytes)
     size_t total;
+};
+
+// Workspace of the fused kernel (bebop_fuse.cu).  A unit is a row pair or a bonus row; a sequence owns
+// `ups` consecutive units (K + 1 for bebop_verify, 1 for bebop_tv); every unit is cut into T slices.
+#ifndef BEBOP_FUSE_WARPS
+#define BEBOP_FUSE_WARPS 16
+#endif
+constexpr int kFuseWarps = BEBOP_FUSE_WARPS;   // consumer warps of a group = warp chunks of a slice
+#ifndef BEBOP_FUSE_VPT
+#define BEBOP_FUSE_VPT 2
+#endif
+constexpr int kFuseSliceVecs = kFuseWarps * 32 * BEBOP_FUSE_VPT;   // 16-byte vectors per slice, at most
+constexpr int kFuseMaxSlices = 128;
+struct FusePlan {
+    int T, slice_vecs;
+    size_t units;
+    // zeroed per call: head (ticket, wait flag, re-draw counters), the re-draw's per-sequence counters, its list, the
+    // per-sequence count of delivered parts, the slice records
+    size_t off_xdone, off_xsdone, off_fbrec, off_seqcnt, off_rec, zero_bytes;
+    size_t off_mass, off_wexp, off_saux, off_smass, off_rows, off_xsum, off_xmass, total;
 };
 
 
@@ -72,6 +93,30 @@ static inline PipePlan make_pipe_plan(int B, int K, int nvec, int dt, int slice_
     return w;
 }
 
+static inline FusePlan make_fuse_plan(int B, int K, int nvec, int ups) {
+    FusePlan f;
+    f.T = (nvec + kFuseSliceVecs - 1) / kFuseSliceVecs; if (f.T < 1) f.T = 1;
+    f.slice_vecs = (nvec + f.T - 1) / f.T;
+    f.units = (size_t)B * (size_t)ups;
+    const PipePlan wv = make_pipe_plan(B, K, nvec, 0);          // the fp64 re-draw cuts rows its own way
+    size_t o = 256;
+    f.off_xdone = o;  o += align256(sizeof(int) * (size_t)B);
+    f.off_xsdone = o; o += align256(sizeof(int) * (size_t)B);
+    f.off_fbrec = o;  o += align256(16 * (size_t)B);
+    f.off_seqcnt = o; o += align256(sizeof(int) * (size_t)B);
+    f.off_rec = o;    o += align256(16 * f.units * f.T * 2);
+    f.zero_bytes = o;
+    f.off_mass = o;   o += align256(8 * f.units * f.T * kFuseWarps);
+    f.off_wexp = o;   o += align256(8 * f.units * f.T * kFuseWarps);
+    f.off_saux = o;   o += align256(8 * f.units * f.T);
+    f.off_smass = o;  o += align256(8 * f.units * f.T);
+    f.off_rows = o;   o += align256(32 * f.units);
+    f.off_xsum = o;   o += align256(16 * (size_t)B * kRedrawCut * wv.T);
+    f.off_xmass = o;  o += align256(8 * (size_t)B * kRedrawCut * wv.T * 8);
+    f.total = o;
+    return f;
+}
+
 static inline Plan make_plan(int B, int K, int V, int dt) {
     Plan p;
     p.B = B; p.K = K; p.V = V; p.dt = dt;
@@ -99,7 +144,11 @@ static inline Plan make_plan(int B, int K, int V, int dt) {
     p.off_dmass = o;  o = align256(o + sizeof(double) * (size_t)B * nsd);
     p.off_amax = o;   o = align256(o + 8 * (size_t)B * (K + 1) * p.nsplit);
     {
-        p.off_pipe = o;   o = align256(o + make_pipe_plan(B, K, p.nvec, dt).total);
+        // one region for the pipelined and the fused kernel: a call runs one of them, and both keep the wait flag
+        // and the re-draw's counters at the same place in its head
+        const size_t wp = make_pipe_plan(B, K, p.nvec, dt).total, wf = make_fuse_plan(B, K, p.nvec, K + 1).total;
+        p.off_pipe = o;
+        p.off_fuse = o;   o = align256(o + (wp > wf ? wp : wf));
     }
     p.total = o;
     return p;

@@ -15,13 +15,14 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-PATHS = {"pipe": 0, "general": 1}
+PATHS = {"pipe": 2, "general": 1, "fuse": 3}
 
 
-@pytest.fixture(autouse=True, params=["pipe", "general"])
+@pytest.fixture(autouse=True, params=["pipe", "general", "fuse"])
 def kernel_path(request):
-    """Every test runs twice: through the pipelined kernel where the shape admits it, and through the
-    general split-row kernels."""
+    """Every test runs three times: through the pipelined kernel and through the fused kernel where the shape admits
+    them, and through the general split-row kernels.  (Left alone, the library picks the faster of the first two for
+    the shape: the other GPU test files run that way.)"""
     P.bebop_debug_force_general_path(PATHS[request.param])
     yield request.param
     P.bebop_debug_force_general_path(0)
@@ -121,7 +122,7 @@ def test_every_sequence_goes_to_the_fp64_redraw(dtype, kernel_path):
     got = run_verify(x)
     got = run_verify(x, workspace=got["workspace"])     # the second call finds the first call's records there
     torch.cuda.synchronize()
-    if kernel_path == "pipe":
+    if kernel_path != "general":
         off = P.bebop_debug_fallback_offset(cfg.B, cfg.K, cfg.V, 0 if dtype == "f32" else 1)
         assert int(got["workspace"][off:off + 4].view(torch.int32).item()) == cfg.B
     check_properties(got, x)

@@ -13,7 +13,7 @@ from parity import TOL, compare_verify, oracle_on, to_np
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-PATHS = {"pipe": 0, "general": 1}
+PATHS = {"pipe": 2, "general": 1, "fuse": 3}
 
 
 def run_verify(x, **kw):
@@ -54,14 +54,16 @@ def test_verify_with_tv_and_without_status_twice_on_one_workspace():
 
 
 # ------------------------------------------------------------------------- bounded waits
+@pytest.mark.parametrize("path", ["pipe", "fuse"])
 @pytest.mark.parametrize("which", [1, 2])
-def test_a_wait_that_runs_out_returns_with_the_status_bit(which):
+def test_a_wait_that_runs_out_returns_with_the_status_bit(which, path):
     """The hook makes one device-side wait give up as if its bound had run out (1: the re-draw kernel's wait for the
-    list of sequences; 2: the producers' wait for a sequence's accept scan).  The call must return, every row must
-    say so, and the next call on the same workspace must be normal again."""
+    list of sequences; 2: the main kernel's wait for what other CTAs deliver -- a sequence's accept scan in the
+    pipelined kernel, a unit's softmax partials in the fused one).  The call must return, every row must say so,
+    and the next call on the same workspace must be normal again."""
     cfg = G.Config("wait", 64, 3, 8192, "bf16", 2.0, True, 1.0, 1.0, seed=63)
     x = G.make_inputs(cfg, DEV)
-    P.bebop_debug_force_general_path(0)
+    P.bebop_debug_force_general_path(PATHS[path])
     ok = run_verify(x)
     torch.cuda.synchronize()
     P.bebop_debug_expire_wait(which)
@@ -74,6 +76,7 @@ def test_a_wait_that_runs_out_returns_with_the_status_bit(which):
     for k in ("accept_len", "out_tokens", "tv", "row_status"):
         assert torch.equal(again[k], ok[k]), k
     compare_verify(again, oracle_on(x), cfg.dtype)
+    P.bebop_debug_force_general_path(0)
 
 
 # ----------------------------------------------------------------------- workspace bounds
@@ -89,11 +92,11 @@ def _intact(buf, nbytes):
     return bool((buf[:GUARD] == 0xA5).all()) and bool((buf[GUARD + nbytes:] == 0xA5).all())
 
 
-@pytest.mark.parametrize("path", ["pipe", "general"])
+@pytest.mark.parametrize("path", ["pipe", "general", "fuse"])
 @pytest.mark.parametrize("dtype,B,K,V", [("f32", 9, 2, 1000), ("bf16", 9, 2, 8), ("bf16", 5, 32, 4096), ("f32", 3, 1, 70001),
                                           ("bf16", 7, 3, 3 * 151936 // 2), ("bf16", 300, 1, 2040)])
 def test_kernels_stay_inside_the_workspace(path, dtype, B, K, V):
-    """4 KB of sentinel bytes before and after exactly bebop_workspace_bytes: every entry point, both paths."""
+    """4 KB of sentinel bytes before and after exactly bebop_workspace_bytes: every entry point, every path."""
     P.bebop_debug_force_general_path(PATHS[path])
     try:
         cfg = G.Config("guard", B, K, V, dtype, 2.0, V >= 16, 0.7, 1.0, ragged=K > 1, seed=64)
@@ -142,11 +145,14 @@ def test_greedy_lowest_index_among_signed_zeros(path):
 
 
 # ------------------------------------------------------------- the fast draw's bound over many seeds
-def test_fast_draw_bound_over_many_seeds_and_temperatures():
+@pytest.mark.parametrize("path", ["pipe", "fuse"])
+def test_fast_draw_bound_over_many_seeds_and_temperatures(path):
     """bebop_verify against the oracle on more than 5,000 sequences at V = 151936: 24 seeds, four temperatures, the
     peaked (rollout) and the flat (high-entropy) recipe, residual and bonus draws.  No unflagged mismatch is allowed,
-    flagged draws stay below 1e-4, and the share of sequences the fp64 re-draw had to decide is reported."""
-    P.bebop_debug_force_general_path(0)
+    flagged draws stay below 1e-4, and the share of sequences the fp64 re-draw had to decide is reported.  Both
+    kernels that keep fast draws: they bound the error in different ways (the pipelined one from the rows' sums of
+    squares, the fused one from the rows' largest probabilities)."""
+    P.bebop_debug_force_general_path(PATHS[path])
     B, K, V = 224, 3, 151936
     seen = flagged = draws = redrawn = bonus = 0
     kappas = (0.0, 0.25, 1.0)                                # how much room the built-in factor 4 leaves
@@ -177,9 +183,10 @@ def test_fast_draw_bound_over_many_seeds_and_temperatures():
                 P.bebop_debug_set_draw_kappa(-1.0)
             kept[kap] += B - int(g2["workspace"][off:off + 4].view(torch.int32).item())
             wrong[kap] += int(((to_np(g2["out_tokens"]) != ref["out_tokens"]).any(axis=1) & ok).sum())
-    print("\nfast-draw bound: %d sequences (%d bonus draws), %d draws, %d flagged by the oracle (%.2e), "
+    P.bebop_debug_force_general_path(0)
+    print("\nfast-draw bound (%s kernel): %d sequences (%d bonus draws), %d draws, %d flagged by the oracle (%.2e), "
           "%d re-drawn in fp64 (%.2f %%), 0 unflagged mismatches"
-          % (seen, bonus, draws, flagged, flagged / draws, redrawn, 100.0 * redrawn / seen))
+          % (path, seen, bonus, draws, flagged, flagged / draws, redrawn, 100.0 * redrawn / seen))
     for kap in kappas:
         print("  factor %.2f: %d of %d draws kept in fp32, %d of them differ from the oracle" % (kap, kept[kap], seen, wrong[kap]))
     assert seen >= 5000 and flagged <= 1e-4 * draws + 1
