@@ -818,7 +818,7 @@ __device__ __forceinline__ int owner_of(const double (&v)[N], double below, doub
 // do not depend on each other are asked for together: the chain is rows and tokens -> the tokens' logits -> accept
 // scan -> slice masses of the draw unit -> chunk masses of the owning slice -> the owning chunk's vectors.
 template <int DT>
-__device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b) {
+__device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, int need) {
     constexpr int VEC = Elem<DT>::VEC;
     constexpr int SPL = kFuseMaxSlices / 32;       // slices per lane, at most
     const RowArgs& R = a.r;
@@ -829,17 +829,42 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b) 
     int seq_st = tau_ok(tau) ? 0 : ST_BAD_TEMP;
     const int unit0 = b * (K + 1);
     const int per = (T + 31) >> 5;                 // a lane's run of slices: [lane * per, lane * per + per)
-    // ---- lane k owns draft position k: its rows, token, uniform
+    // ---- lane k owns draft position k: its token, uniform and the token's logits are the call's inputs, asked for
+    // before the wait for the sequence's parts
     const bool active = lane < L;
     const int tk = active ? a.draft_tokens[(int64_t)b * K + lane] : 0;
     const float u = active ? a.u_accept[(int64_t)b * K + lane] : 0.f;
-    FRow sp, sq;
-    sp.inv_s = 0.0; sp.e = E_EMPTY; sp.st = 0; sq = sp;
-    if (active) { sp = ld_row(a.rows + 2 * (int64_t)(unit0 + lane)); sq = ld_row(a.rows + 2 * (int64_t)(unit0 + lane) + 1); }
-    // ---- TV of every position: the sum of its slice masses, in slice order (asked for now, used after the scan)
+    const float uf = a.u_final[b];
     const bool tok_ok = tk >= 0 && tk < V;
     float zpx = 0.f, zqx = 0.f;
     if (active && tok_ok) { zpx = load_one<DT>(row_ptr(R, b, lane), tk); zqx = load_one<DT>(row_ptr(R, b, K + 1 + lane), tk); }
+    if (!wait_parts(a, S, b, need)) {
+        // the parts never came: the sequence gets no draw (the re-draw kernel must not wait for it) and says so
+        if (lane == 0) {
+            atomicExch(a.wait_failed, 1);
+            a.o.accept_len[b] = 0;
+            for (int q = 0; q <= K; ++q) a.o.out_tokens[(int64_t)b * (K + 1) + q] = -1;
+            if (a.o.row_status) a.o.row_status[b] = ST_WAIT;
+            draw_decided(a.fb_count);
+        }
+        return;
+    }
+    // ---- its rows
+    FRow sp, sq;
+    sp.inv_s = 0.0; sp.e = E_EMPTY; sp.st = 0; sq = sp;
+    if (active) { sp = ld_row(a.rows + 2 * (int64_t)(unit0 + lane)); sq = ld_row(a.rows + 2 * (int64_t)(unit0 + lane) + 1); }
+    // ---- TV of every position: the slices' masses, asked for now four positions at a time, summed after the scan
+    constexpr int TVG = 4;
+    double tvz[TVG];
+#pragma unroll
+    for (int g = 0; g < TVG; ++g) {
+        tvz[g] = 0.0;
+        if (a.o.tv && g < L) {
+            const double* m = a.smass + (int64_t)(unit0 + g) * T + lane * per;
+#pragma unroll
+            for (int i = 0; i < SPL; ++i) if (i < per && lane * per + i < T) tvz[g] += __ldcg(m + i);
+        }
+    }
     if (!seq_st && __ballot_sync(0xffffffffu, active && !tok_ok)) seq_st = ST_BAD_TOKEN;
     const int rs = active ? (sp.st | sq.st) : 0;
     const unsigned badrows = __ballot_sync(0xffffffffu, rs != 0);
@@ -906,7 +931,14 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b) 
     if (fatal) { if (lane == 0) draw_decided(a.fb_count); return; }
     // ---- TV of every position: the sum of its slices' masses (slice order within a lane, lanes in a fixed tree)
     if (a.o.tv) {
-        for (int k = 0; k < L; ++k) {
+#pragma unroll
+        for (int g = 0; g < TVG; ++g) {
+            if (g < L) {
+                const double z = warp_sum(tvz[g]);
+                if (lane == 0) a.o.tv[(int64_t)b * K + g] = (float)fmin(fmax(z, 0.0), 1.0);
+            }
+        }
+        for (int k = TVG; k < L; ++k) {
             const double* m = a.smass + (int64_t)(unit0 + k) * T + lane * per;
             double z = 0.0;
 #pragma unroll
@@ -935,7 +967,7 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b) 
     // the total as the scan below adds it up, so that u = 1 lands inside the last slice
     double sbase, Zs;
     owner_of<SPL>(sm, 0.0, -1.0, &sbase, &Zs);
-    const double Tt = (double)a.u_final[b] * Zs;
+    const double Tt = (double)uf * Zs;
     int y = -1, cert = 0;
     const int lane_s = Tt > 0.0 ? owner_of<SPL>(sm, 0.0, Tt, &sbase, &Zs) : -1;      // lane-major index -> slice
     if (lane_s >= 0) {
@@ -1020,23 +1052,10 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b) 
 template <int DT, bool TVM>
 __device__ __forceinline__ void f_finish(const FuseArgs& a, FShared& S, unsigned char* scratch, int w) {
     const RowArgs& R = a.r;
-    const int lane = threadIdx.x & 31;
     (void)scratch;
     for (int b = w * (int)gridDim.x + (int)blockIdx.x; b < R.B; b += FCW * (int)gridDim.x) {
         if (TVM) { f_finish_tv(a, S, b); continue; }
-        const int need = len_of(R, b) * a.T + (a.T + 1) / 2;
-        if (!wait_parts(a, S, b, need)) {
-            // the parts never came: the sequence gets no draw (the re-draw kernel must not wait for it) and says so
-            if (lane == 0) {
-                atomicExch(a.wait_failed, 1);
-                a.o.accept_len[b] = 0;
-                for (int q = 0; q <= R.K; ++q) a.o.out_tokens[(int64_t)b * (R.K + 1) + q] = -1;
-                if (a.o.row_status) a.o.row_status[b] = ST_WAIT;
-                draw_decided(a.fb_count);
-            }
-            continue;
-        }
-        f_finish_seq<DT>(a, S, b);
+        f_finish_seq<DT>(a, S, b, len_of(R, b) * a.T + (a.T + 1) / 2);
         __syncwarp();
     }
 }
