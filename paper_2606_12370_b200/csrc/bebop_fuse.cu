@@ -817,10 +817,9 @@ __device__ __forceinline__ int owner_of(const double (&v)[N], double below, doub
 // One warp; everything it reads was published before the sequence's count reached its final value.  The loads that
 // do not depend on each other are asked for together: the chain is rows and tokens -> the tokens' logits -> accept
 // scan -> slice masses of the draw unit -> chunk masses of the owning slice -> the owning chunk's vectors.
-template <int DT>
+template <int DT, int SPL>                         // SPL: slices per lane, at most
 __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, int need) {
     constexpr int VEC = Elem<DT>::VEC;
-    constexpr int SPL = kFuseMaxSlices / 32;       // slices per lane, at most
     const RowArgs& R = a.r;
     const int lane = threadIdx.x & 31;
     const int K = R.K, V = R.V, T = a.T, L = len_of(R, b);
@@ -932,12 +931,12 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
     // ---- TV of every position: the sum of its slices' masses (slice order within a lane, lanes in a fixed tree)
     if (a.o.tv) {
 #pragma unroll
-        for (int g = 0; g < TVG; ++g) {
-            if (g < L) {
-                const double z = warp_sum(tvz[g]);
-                if (lane == 0) a.o.tv[(int64_t)b * K + g] = (float)fmin(fmax(z, 0.0), 1.0);
-            }
-        }
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int g = 0; g < TVG; ++g) tvz[g] += shfl_xor_d(tvz[g], o);
+#pragma unroll
+        for (int g = 0; g < TVG; ++g)
+            if (g < L && lane == 0) a.o.tv[(int64_t)b * K + g] = (float)fmin(fmax(tvz[g], 0.0), 1.0);
         for (int k = TVG; k < L; ++k) {
             const double* m = a.smass + (int64_t)(unit0 + k) * T + lane * per;
             double z = 0.0;
@@ -1055,7 +1054,10 @@ __device__ __forceinline__ void f_finish(const FuseArgs& a, FShared& S, unsigned
     (void)scratch;
     for (int b = w * (int)gridDim.x + (int)blockIdx.x; b < R.B; b += FCW * (int)gridDim.x) {
         if (TVM) { f_finish_tv(a, S, b); continue; }
-        f_finish_seq<DT>(a, S, b, len_of(R, b) * a.T + (a.T + 1) / 2);
+        const int need = len_of(R, b) * a.T + (a.T + 1) / 2;
+        if (a.T <= 32) f_finish_seq<DT, 1>(a, S, b, need);
+        else if (a.T <= 64) f_finish_seq<DT, 2>(a, S, b, need);
+        else f_finish_seq<DT, kFuseMaxSlices / 32>(a, S, b, need);
         __syncwarp();
     }
 }
