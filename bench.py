@@ -48,7 +48,7 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-KERNEL_OF_PATH = {0: "k_pipe"}
+KERNEL_NAME = {1: "general kernels", 2: "k_pipe", 3: "k_fuse"}      # by bebop_debug_last_kernel()
 
 
 def ncu_traffic(kernel):
@@ -288,6 +288,7 @@ def config_line(torch, P, G, name, dev, barrier, calls):
     got_len, got_tok = out["accept_len"][sel].cpu().numpy(), out["out_tokens"][sel].cpu().numpy()
     differ = (got_len != ref["accept_len"]) | (got_tok != ref["out_tokens"]).any(axis=1)
     line = {"shape": "B=%d K=%d V=%d %s%s" % (B, K, V, cfg.dtype, " ragged" if cfg.ragged else ""),
+            "kernel": KERNEL_NAME.get(P.bebop_debug_last_kernel()),
             "ms_per_call": st, "positions_per_s": positions / (st["mean"] * 1e-3),
             "algorithmic_bytes": alg, "algorithmic_gbs": alg / (st["mean"] * 1e-3) / 1e9,
             "pct_of_8tbs": 100.0 * alg / (st["mean"] * 1e-3) / 1e9 / NORTH_STAR_PEAK_GBS,
@@ -400,7 +401,8 @@ def run_ours(args):
     kern_ms = [a_.elapsed_time(b_) for a_, b_ in pairs]
     kern_ms = sum(kern_ms) / len(kern_ms)
     clocks = sampler.summary(t0, t1)
-    launches_per_call = 6 if args.path == 1 else 2      # main kernel, fp64 re-draw kernel | 6 general kernels
+    main_kernel = P.bebop_debug_last_kernel()           # what the timed calls ran: the library chooses by shape
+    launches_per_call = 6 if main_kernel == 1 else 2    # main kernel, fp64 re-draw kernel | 6 general kernels
 
     # median and best of single calls (an event pair around each call, so a little above the back-to-back mean)
     single = stats(per_call_ms(torch, [step], max(10, min(steps, 100)), barrier))
@@ -432,11 +434,13 @@ def run_ours(args):
     # the two other entry points on the same logits (reported beside the headline, not part of it)
     other_steps = max(1, min(steps, 50))
     tv_ms = gr_ms = float("nan")
+    tv_kernel = 0
     if x["draft_len"] is None:
         tv_t = x["target"][:, :K].reshape(B * K, V)
         tv_d = x["draft"].reshape(B * K, V)
         tvws = torch.empty(P.bebop_workspace_bytes(B * K, 1, V, P.BEBOP_BF16), dtype=torch.uint8, device=dev)
         tv_ms = timed(lambda: P.bebop_tv(tv_t, tv_d, temperature_all=1.0, workspace=tvws), other_steps)
+        tv_kernel = P.bebop_debug_last_kernel()
         gr_ms = timed(lambda: P.bebop_greedy_verify(x["target"], x["draft_tokens"], workspace=ws), other_steps)
 
     # end to end: pinned host inputs -> device, same C-ABI call, results back to the host
@@ -502,7 +506,7 @@ def run_ours(args):
             "gpu_launches": steps * launches_per_call,
             "single_call_ms": single,
             "other_entry_points": {
-                "bebop_tv": {"ms_per_call": tv_ms, "row_pairs": world * B * K, "steps": other_steps,
+                "bebop_tv": {"ms_per_call": tv_ms, "row_pairs": world * B * K, "steps": other_steps, "kernel": KERNEL_NAME.get(tv_kernel),
                              "algorithmic_gbs": world * B * K * 2 * V * es / (tv_ms * 1e-3) / 1e9},
                 "bebop_greedy_verify": {"ms_per_call": gr_ms, "steps": other_steps,
                                         "algorithmic_gbs": world * B * (K + 1) * V * es / (gr_ms * 1e-3) / 1e9}},
@@ -511,7 +515,7 @@ def run_ours(args):
             "hbm_gbs": gbs, "hbm_pct_of_8tbs": 100.0 * gbs / NORTH_STAR_PEAK_GBS,
             "target": "70 % of 8 TB/s for the fused kernel (north star): not met",
             "input_checksums": checksums(G, x),
-            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, headline, KERNEL_OF_PATH.get(args.path, "general kernels"), len(pairs)),
+            "roofline": roofline(alg_bytes, kern_ms, peak, peak_kind, headline, KERNEL_NAME.get(main_kernel, "general kernels"), len(pairs)),
         }
         if world == 1 and not args.no_configs:
             del host, dev_in, staged
@@ -567,7 +571,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: sequences per GPU instead of the workload's 256 (not a bench line)")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
-    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default: pipelined kernel, 1 general kernels)")
+    ap.add_argument("--path", type=int, default=0, help="profiling aid: kernel path (0 default: chosen by shape, 1 general kernels, 2 pipelined kernel, 3 fused kernel)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # no launcher: start the ranks here, one per GPU

@@ -166,7 +166,8 @@ bebop_status_t bebop_greedy_verify(
  * 0 (the default) the faster, by measurement, of the fused and the pipelined kernel for the shape, and the
  * split-row general kernels for shapes neither takes; 1 the general kernels always; 2 never the fused kernel;
  * 3 the fused kernel wherever it applies (the greedy mode has no fused form).  All give the same results up to
- * the documented tolerances.
+ * the documented tolerances.  bebop_debug_last_kernel() says what the last of these calls ran: 1 the general kernels,
+ * 2 the pipelined kernel, 3 the fused kernel (0: no call yet).
  * bebop_debug_fallback_offset returns the byte offset, inside the workspace of this
  * shape, of an int32 that after a bebop_verify call holds the number of sequences
  * whose draw was re-done by the fp64 kernels.
@@ -182,6 +183,7 @@ bebop_status_t bebop_greedy_verify(
  * 0 keeps every fp32 draw).  For the test that shows how much room the built-in value leaves.
  */
 void bebop_debug_force_general_path(int on);
+int bebop_debug_last_kernel(void);
 size_t bebop_debug_fallback_offset(int B, int K, int V, bebop_dtype_t dt);
 void bebop_debug_set_timing_events(void* start, void* stop);
 void bebop_debug_expire_wait(int which);

@@ -51,6 +51,8 @@ def load_library():
     lib.bebop_debug_force_general_path.argtypes = [i32]
     lib.bebop_debug_set_timing_events.restype = None
     lib.bebop_debug_set_timing_events.argtypes = [vp, vp]
+    lib.bebop_debug_last_kernel.restype = C.c_int
+    lib.bebop_debug_last_kernel.argtypes = []
     lib.bebop_debug_set_draw_kappa.restype = None
     lib.bebop_debug_set_draw_kappa.argtypes = [f32]
     lib.bebop_debug_expire_wait.restype = None
@@ -97,6 +99,11 @@ def _rows(t: torch.Tensor, ndim: int):
 
 def bebop_debug_force_general_path(on) -> None:
     load_library().bebop_debug_force_general_path(int(on))
+
+
+def bebop_debug_last_kernel() -> int:
+    """What the last bebop_verify / bebop_tv / bebop_greedy_verify call ran: 1 general kernels, 2 pipelined kernel, 3 fused kernel."""
+    return int(load_library().bebop_debug_last_kernel())
 
 
 def bebop_debug_set_draw_kappa(kappa) -> None:

@@ -9,6 +9,7 @@ namespace {
 
 // Test hook: route bebop_verify through the general (split-row) path even where the fused
 // kernel applies, so that both paths are covered by the parity tests.
+int g_last_kernel = 0;   // what the last call ran: 1 general kernels, 2 pipelined kernel, 3 fused kernel
 int g_path = 0;   // 0: the faster of the fused and the pipelined kernel where they apply, else the general kernels;
                   // 1: general kernels only; 2: never the fused kernel; 3: the fused kernel wherever it applies
 
@@ -111,10 +112,15 @@ bebop_status_t bebop_verify(const void* target_logits, int64_t ld_target, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, false))) && fuse_supported(a))
+    g_last_kernel = 1;
+    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, false))) && fuse_supported(a)) {
         e = fuse_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
-    if (e == cudaSuccess && !launched && g_path != 1 && pipe_supported(a))
+        if (launched) g_last_kernel = 3;
+    }
+    if (e == cudaSuccess && !launched && g_path != 1 && pipe_supported(a)) {
         e = pipe_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream, &launched);
+        if (launched) g_last_kernel = 2;
+    }
     if (e == cudaSuccess && !launched) e = general_verify(a, p, draft_tokens, u_accept, u_final, o, ws, stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
 }
@@ -139,11 +145,15 @@ bebop_status_t bebop_tv(const void* target_logits, int64_t ld_target, const void
     cudaError_t e = cudaSuccess;
     bool launched = false;
     VerifyOut o{nullptr, nullptr, tv, nullptr, nullptr, row_status};
-    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, true))) && fuse_supported(a))
+    g_last_kernel = 1;
+    if ((g_path == 3 || (g_path == 0 && fuse_preferred(a, true))) && fuse_supported(a)) {
         e = fuse_verify(a, p, nullptr, nullptr, nullptr, o, static_cast<char*>(workspace), stream, &launched, true, s_aux);
+        if (launched) g_last_kernel = 3;
+    }
     if (e == cudaSuccess && !launched && g_path != 1 && pipe_supported(a)) {
         // the pipelined kernel with row pairs in place of sequences: first sweep, second sweep, no draw
         e = pipe_verify(a, p, nullptr, nullptr, nullptr, o, static_cast<char*>(workspace), stream, &launched, true, s_aux);
+        if (launched) g_last_kernel = 2;
     }
     if (e == cudaSuccess && !launched)
         e = general_tv(a, p, tv, s_aux, row_status, static_cast<char*>(workspace), stream);
@@ -168,8 +178,11 @@ bebop_status_t bebop_greedy_verify(const void* target_logits, int64_t ld_target,
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaSuccess;
     bool launched = false;
-    if (g_path != 1 && pipe_supported(a))
+    g_last_kernel = 1;
+    if (g_path != 1 && pipe_supported(a)) {
         e = pipe_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream, &launched);
+        if (launched) g_last_kernel = 2;
+    }
     if (e == cudaSuccess && !launched)
         e = general_greedy(a, p, draft_tokens, accept_len, out_tokens, row_status, static_cast<char*>(workspace), stream);
     return e == cudaSuccess ? BEBOP_OK : BEBOP_ERR_CUDA;
@@ -209,6 +222,8 @@ bebop_status_t bebop_tv_static(const void* target_logits, int64_t ld_target, con
 }
 
 void bebop_debug_force_general_path(int on) { g_path = on; }
+
+int bebop_debug_last_kernel(void) { return g_last_kernel; }
 
 void bebop_debug_expire_wait(int which) { g_expire_wait = which; }
 

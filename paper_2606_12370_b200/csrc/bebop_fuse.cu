@@ -1137,14 +1137,15 @@ bool fuse_supported(const RowArgs& a) {
 // (the merge of a unit's records then takes several records per lane).  bebop_verify is faster up to about ten slices per row
 // (7 per cent at 65,536 bf16 logits, 15 at 32,768, twice as fast at 16,384 and below) and 3 to 8 per cent slower
 // from 100,000 on, where the pipelined kernel streams at close to the copy rate; small calls (a few dozen tasks per
-// CTA) are faster fused at any row length.
+// CTA) are faster fused at any row length, tiny ones (fewer than two tasks per SM) through the pipelined kernel.
 bool fuse_preferred(const RowArgs& a, bool tv_only) {
     const int T = make_fuse_plan(a.B, a.K, a.nvec, 1).T;
-    if (tv_only) return T <= 32;
-    if (T <= 10) return true;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return false; }
-    return T <= 32 && (long long)a.B * (a.K + 1) * T <= 40LL * sms;
+    const long long tasks = (long long)a.B * (tv_only ? 1 : a.K + 1) * T;
+    if (T > 32 || tasks < 2LL * sms) return false;       // (a call of a few tasks is all start-up: 0.038 against 0.031 ms)
+    if (tv_only || T <= 10) return true;
+    return tasks <= 40LL * sms;
 }
 
 cudaError_t fuse_verify(const RowArgs& a, const Plan& p, const int32_t* draft_tokens, const float* u_accept,

@@ -191,3 +191,22 @@ def test_fast_draw_bound_over_many_seeds_and_temperatures(path):
         print("  factor %.2f: %d of %d draws kept in fp32, %d of them differ from the oracle" % (kap, kept[kap], seen, wrong[kap]))
     assert seen >= 5000 and flagged <= 1e-4 * draws + 1
     assert wrong[1.0] == 0, "a quarter of the built-in factor already lets a wrong token through"
+
+
+# ------------------------------------------------------------------ which kernel runs
+def test_the_library_chooses_the_kernel_by_shape():
+    """Left alone, bebop_tv goes through the fused kernel (up to 32 slices per row), bebop_verify through the fused
+    kernel on small vocabularies and small calls and through the pipelined kernel on large ones; the hook overrides."""
+    P.bebop_debug_force_general_path(0)
+    small = G.make_inputs(G.Config("d1", 400, 3, 8192, "bf16", 2.0, True, 1.0, 1.0, seed=71), DEV)
+    large = G.make_inputs(G.Config("d2", 200, 3, 151936, "bf16", 2.0, True, 1.0, 1.0, seed=72), DEV)
+    run_verify(small); assert P.bebop_debug_last_kernel() == 3
+    run_verify(large); assert P.bebop_debug_last_kernel() == 2
+    P.bebop_tv(large["target"][:, 0], large["draft"][:, 0]); assert P.bebop_debug_last_kernel() == 3
+    P.bebop_greedy_verify(large["target"], large["draft_tokens"]); assert P.bebop_debug_last_kernel() == 2
+    for mode, want in ((1, 1), (2, 2), (3, 3), (0, 3)):
+        P.bebop_debug_force_general_path(mode)
+        run_verify(small)
+        assert P.bebop_debug_last_kernel() == want
+    P.bebop_debug_force_general_path(0)
+    torch.cuda.synchronize()
