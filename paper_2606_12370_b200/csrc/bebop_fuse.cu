@@ -1,9 +1,9 @@
 // Fused kernel: bebop_verify and bebop_tv with every logit row read from memory once and exponentiated once.
 //
-// A row (pair) is cut into T slices of at most FSV 16-byte vectors; a task is one slice of one unit, a unit
-// being a row pair (target row k, draft row k of a sequence) or a sequence's bonus row.  Tasks are dealt round
-// robin over a grid that is resident as a whole (one CTA per SM), so the T slices of a unit are in the hands
-// of T different CTAs at about the same time.  Per task, a CTA
+// A row (pair) is cut into T slices of at most FSV 16-byte vectors; a task is one slice of a row pair (target row
+// k, draft row k of a sequence: a "unit") or two slices of a sequence's bonus row.  Tasks are dealt round robin
+// over a grid that is resident as a whole (one CTA per SM), so the T slices of a unit are in the hands of T
+// different CTAs at about the same time.  Per task, a CTA
 //   pass 1  takes the slice from shared memory (bulk copies, a ring of stages), forms e = 2^(x c - E) around an
 //           integer reference exponent E per warp, parks the e of both rows in TENSOR MEMORY (this path has no
 //           contraction, so the 256 KB of TMEM per SM are free to serve as a store), and publishes the
@@ -13,17 +13,16 @@
 //   pass 2  (three tasks behind pass 1: the depth of the TMEM ring hides the exchange) takes its e back from
 //           TMEM and forms r' = max(0, e_p - rho e_q), rho = S_p / S_q as two floats scaled to the warp's
 //           exponents: the residual p - q up to the factor 1 / S_p, which is applied once per warp chunk, in
-//           double.  The chunk masses give TV (their sum) and the inverse CDF of the draw (it walks them); with
-//           them go the sum of squares the draw's error bound needs and, for bebop_tv, the auxiliary sum of
-//           Eq. tv_grad.
+//           double.  The chunk and slice masses give TV (their sum) and the inverse CDF of the draw (it walks
+//           them); for bebop_tv the auxiliary sum of Eq. tv_grad goes with them.
 // The consumer warps neither shuffle nor wait for each other: a thread leaves its partial sums in shared
-// memory and publisher warps add them up in double.  When a CTA has run out of tasks, its consumer warps
-// complete sequences, one warp each: merge the rows, run the accept scan (Algorithm 3), write TV, locate the
-// warp chunk that owns the target u Z of the inverse CDF, evaluate that chunk's tokens again and keep the token
-// if the crossing clears the error bound; else the sequence is listed for the fp64 re-draw kernel.
+// memory and publisher warps add them up.  When a CTA has run out of tasks, its consumer warps complete
+// sequences, one warp each: run the accept scan (Algorithm 3) on the merged rows, write TV, locate the slice and
+// the warp chunk that own the target u Z of the inverse CDF, evaluate that chunk's tokens again and keep the
+// token if the crossing clears the error bound; else the sequence is listed for the fp64 re-draw kernel.
 //
-// Warps: 16 consumers, producer, publisher of the softmax partials, publisher of the masses, four stats warps
-// (stats warp j serves the tasks n = j mod 4, so that the latency of one merge does not bound the task rate).
+// Warps: 16 consumers, producer, publisher of the softmax partials, two publishers of the masses, four stats
+// warps (stats warp j serves the tasks n = j mod 4, so that the latency of one merge does not bound the task rate).
 // What CTAs pass to each other: records of two 8-byte words, each word valid by itself once non-zero (the memory
 // is zeroed per call), written and read by relaxed 64-bit accesses; and the per-sequence count of delivered
 // parts, added after a fence and read with acquire.  Every wait is bounded and sleeps between looks (a waiting
@@ -1049,9 +1048,8 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
 
 // consumer warp w of CTA i completes the sequences w * grid + i, then every 16 * grid further on
 template <int DT, bool TVM>
-__device__ __forceinline__ void f_finish(const FuseArgs& a, FShared& S, unsigned char* scratch, int w) {
+__device__ __forceinline__ void f_finish(const FuseArgs& a, FShared& S, int w) {
     const RowArgs& R = a.r;
-    (void)scratch;
     for (int b = w * (int)gridDim.x + (int)blockIdx.x; b < R.B; b += FCW * (int)gridDim.x) {
         if (TVM) { f_finish_tv(a, S, b); continue; }
         const int need = len_of(R, b) * a.T + (a.T + 1) / 2;
@@ -1085,9 +1083,7 @@ __global__ void __launch_bounds__(FT, 1) k_fuse(const __grid_constant__ FuseArgs
     const uint32_t tmem0 = S.tmem_base;
     if (warp < FCW) {
         f_consumer<DT, TVM>(a, S, smem, tid);
-        // the ring of stages is free once every consumer warp has left the loop: it serves as scratch now
-        asm volatile("bar.sync 1, %0;" :: "n"(FCT) : "memory");
-        f_finish<DT, TVM>(a, S, smem, warp);
+        f_finish<DT, TVM>(a, S, warp);
     }
     else if (warp == W_PROD) { if ((tid & 31) == 0) f_producer<DT>(a, S, smem, total); __syncwarp(); }
     else if (warp == W_PUBA) f_puba(a, S);
