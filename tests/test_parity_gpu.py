@@ -270,6 +270,28 @@ def test_tv_entry_point(dtype, V):
     np.testing.assert_array_equal(to_np(got["row_status"]), ref["row_status"])
 
 
+@pytest.mark.parametrize("dtype,N,V", [("bf16", 20000, 8), ("f32", 9001, 40), ("bf16", 3000, 2056)])
+def test_tv_many_short_rows(dtype, N, V):
+    """More row pairs than there are warps to complete them (every warp completes several), rows of one slice,
+    some of them masked, empty or poisoned, per-row temperatures."""
+    gen = torch.Generator(device=DEV).manual_seed(77)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    tgt = (2.0 * torch.randn(N, V, generator=gen, device=DEV)).to(tdt)
+    drf = (tgt.float() + 0.8 * torch.randn(N, V, generator=gen, device=DEV)).to(tdt)
+    tgt[5, V // 2:] = float("-inf")
+    drf[6, :] = float("-inf")                  # an empty draft row
+    tgt[7, 3] = float("nan")
+    drf[N - 1, :] = tgt[N - 1, :]              # the last row pair: identical rows
+    temp = 0.6 + 0.6 * torch.rand(N, generator=gen, device=DEV)
+    got = P.bebop_tv(tgt, drf, temperature=temp)
+    ref = oracle.tv(tgt.float().cpu().numpy(), drf.float().cpu().numpy(), temperature=to_np(temp))
+    np.testing.assert_array_equal(to_np(got["row_status"]), ref["row_status"])
+    ok = ref["row_status"] == 0
+    assert np.abs(to_np(got["tv"]) - ref["tv"])[ok].max() <= TOL[dtype]
+    assert np.abs(to_np(got["s_aux"]) - ref["s_aux"])[ok].max() <= TOL[dtype]
+    assert float(got["tv"][N - 1]) == 0.0
+
+
 # ---------------------------------------------------------------------- greedy
 @pytest.mark.parametrize("dtype,V,K", [("f32", 1000, 3), ("bf16", 151936, 3), ("bf16", 8, 1), ("bf16", 4096, 32)])
 def test_greedy_entry_point(dtype, V, K):
