@@ -1180,12 +1180,20 @@ cudaError_t fuse_verify(const RowArgs& a, const Plan& p, const int32_t* draft_to
     const int grid = (int)(total < grid_max ? total : grid_max);
     if (grid < fp.T) return cudaSuccess;
     if (g_ev_start) cudaEventRecord(g_ev_start, stream);
-    if (tv_only) {
-        if (a.dt == 0) k_fuse<0, true><<<grid, FT, kFuseSmem, stream>>>(fa, (int)total);
-        else k_fuse<1, true><<<grid, FT, kFuseSmem, stream>>>(fa, (int)total);
-    } else {
-        if (a.dt == 0) k_fuse<0, false><<<grid, FT, kFuseSmem, stream>>>(fa, (int)total);
-        else k_fuse<1, false><<<grid, FT, kFuseSmem, stream>>>(fa, (int)total);
+    {
+        // A cooperative launch: the device takes the grid only as a whole, so CTAs of two such grids (two streams) cannot
+        // end up holding SMs while each waits for partners that found no room.
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(FT); cfg.dynamicSmemBytes = kFuseSmem; cfg.stream = stream;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const int tot = (int)total;
+        if (tv_only) e = a.dt == 0 ? cudaLaunchKernelEx(&cfg, k_fuse<0, true>, fa, tot) : cudaLaunchKernelEx(&cfg, k_fuse<1, true>, fa, tot);
+        else e = a.dt == 0 ? cudaLaunchKernelEx(&cfg, k_fuse<0, false>, fa, tot) : cudaLaunchKernelEx(&cfg, k_fuse<1, false>, fa, tot);
+        if (e == cudaErrorCooperativeLaunchTooLarge) { cudaGetLastError(); return cudaSuccess; }     // no room for the whole grid: the caller takes the pipelined kernel
+        if (e != cudaSuccess) return e;
     }
     e = cudaGetLastError();
     if (g_ev_stop) cudaEventRecord(g_ev_stop, stream);
