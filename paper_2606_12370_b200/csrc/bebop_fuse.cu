@@ -624,8 +624,10 @@ __device__ __forceinline__ void f_puba(const FuseArgs& a, FShared& S) {
 
 // ------------------------------------------------------------------ publisher of the masses
 // Publisher j serves the iterations n = j mod FNPB.  Pair tasks: the chunks' sums of r' times 2^(E_wp - E_p) / S_p
-// are the chunks' residual masses; with them the warps' exponents and the slice's auxiliary sum.  Then one count for the sequence, behind a
-// fence: who sees the count sees the parts.  Pass 2 of task m is in place after iteration m + FLAG.
+// are the chunks' residual masses; with them go the warps' exponents, the slice's mass and auxiliary sum and, with
+// slice 0, the unit's merged rows.  Bonus tasks: the chunk sums the other publisher left.  Then one count for the
+// sequence, behind a fence: who sees the count sees the parts.  Pass 2 of task m is in place after iteration
+// m + FLAG.
 template <bool TVM>
 __device__ __forceinline__ void f_pubb(const FuseArgs& a, FShared& S, int j) {
     const int lane = threadIdx.x & 31;
