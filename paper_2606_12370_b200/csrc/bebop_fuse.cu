@@ -79,8 +79,12 @@ struct __align__(16) FTask {
 // what the publication of a task's pass 2 needs: the rows' exponents and normalisers
 struct __align__(16) FScale { double inv_p, inv_q; int ep, eq; float rho_h, rho_l; int stp, stq, pad0, pad1; };
 struct __align__(16) FWarpE { int ep, eq, flags, pad; };               // a consumer warp's exponents of a task
-// softmax partial of one slice of one row; each 8-byte word is valid by itself once non-zero
+// Softmax partial of one slice of one row; each 8-byte word is valid by itself once non-zero.  `flags`: bit 0 says
+// that the slice holds a NaN or +inf; the other bits are those of a float u, with which the slice's sum of e^2
+// (around the slice's exponent) is at most sqrt(2) u: u = sum over the warp chunks of 4^(E_w - E_s) times the
+// chunk's sum of e, as the e of a chunk are at most sqrt(2) around the chunk's own exponent.
 struct __align__(16) FRec { double s; int ecode; int flags; };
+__device__ __forceinline__ float rec_ub(const FRec& r) { return __int_as_float(r.flags & ~1); }
 struct __align__(16) FRow { double inv_s; int e; int st; };           // a merged row: 1/S, exponent, status bits
 struct FRho { float h, l; };
 
@@ -275,7 +279,7 @@ __device__ __forceinline__ void merge_rows_n(const FuseArgs& a, FShared& S, int 
 #pragma unroll
     for (int i = 0; i < SPL; ++i)
 #pragma unroll
-        for (int w = 0; w < 2; ++w) { el[w] = max(el[w], (r[i][w].ecode - 1) >> 1); fl |= r[i][w].flags << w; }
+        for (int w = 0; w < 2; ++w) { el[w] = max(el[w], (r[i][w].ecode - 1) >> 1); fl |= (r[i][w].flags & 1) << w; }
     const int Em[2] = {redux_max(el[0]), redux_max(el[1])};
     fl = __reduce_or_sync(0xffffffffu, fl);
     double v[2] = {0.0, 0.0};
@@ -596,9 +600,11 @@ __device__ __forceinline__ void f_puba(const FuseArgs& a, FShared& S) {
         // role 0: the target row; role 1: the draft row.  A chunk's sum is below 2^11, its scaling a power of two.
         const bool second = role == 1;
         const int ew = second ? we.eq : we.ep, em = second ? emq : emp;
-        double v = ew > E_EMPTY ? (double)(second ? sc2.y : sc2.x) * pow2d(max(ew - em, -1000)) : 0.0;
+        const double f = ew > E_EMPTY ? pow2d(max(ew - em, -500)) : 0.0;
+        double v = (double)(second ? sc2.y : sc2.x) * f;
+        double ub = v * f;                                  // 4^(E_w - E_s) times the chunk's sum of e
 #pragma unroll
-        for (int o = 16; o >= FLPC; o >>= 1) v += shfl_xor_d(v, o);
+        for (int o = 16; o >= FLPC; o >>= 1) { v += shfl_xor_d(v, o); ub += shfl_xor_d(ub, o); }
         {
             // Every lane forms the record; lanes 0 and (for a pair) 1 store it, by predicate.  As a branch for those two
             // lanes the store came about a microsecond late: nothing makes a warp that has split reconverge before
@@ -607,7 +613,9 @@ __device__ __forceinline__ void f_puba(const FuseArgs& a, FShared& S) {
             double rs = em > E_EMPTY && !bad ? v : 0.0;
             if (rs == 0.0) rs = -0.0;
             const unsigned long long w0 = (unsigned long long)__double_as_longlong(rs);
-            const unsigned long long w1 = (unsigned long long)(unsigned)(2 * em + 1) | ((unsigned long long)(bad ? 1u : 0u) << 32);
+            // (the bound rounded up, and up again to an even bit pattern: bit 0 of the word is the flag)
+            const unsigned ubits = ((unsigned)__float_as_int(__double2float_ru((em > E_EMPTY && !bad) ? ub : 0.0)) + 1u) & ~1u;
+            const unsigned long long w1 = (unsigned long long)(unsigned)(2 * em + 1) | ((unsigned long long)(ubits | (bad ? 1u : 0u)) << 32);
             const bool two = pair || d.s + 1 < a.T;            // a second record: the draft row's, or the bonus row's second slice's
             const unsigned doit = (lane == 0 || (lane == 1 && two)) ? 1u : 0u;
             asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};\n\t}"
@@ -883,9 +891,9 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
     const int n = rej ? __ffs(rej) - 1 : L;
     // ---- the bonus row, when every draft was accepted: merged here from its slices' records (kept: they are its masses)
     FRow rb; rb.inv_s = 0.0; rb.e = E_EMPTY; rb.st = 0;
-    double bs[SPL]; int be[SPL];
+    double bs[SPL], bu[SPL]; int be[SPL];
 #pragma unroll
-    for (int i = 0; i < SPL; ++i) { bs[i] = 0.0; be[i] = E_EMPTY; }
+    for (int i = 0; i < SPL; ++i) { bs[i] = 0.0; bu[i] = 0.0; be[i] = E_EMPTY; }
     if (!(seq_st & ST_FATAL) && n == L) {
         const FRec* base = a.rec + ((int64_t)(unit0 + L) * T) * 2;
         int fl = 0, el = E_EMPTY;
@@ -897,7 +905,7 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
                 bool ok = ld_rec(base + 2 * si, &r);
                 for (uint32_t it = 0; !ok && it < kSpin; ++it) { __nanosleep(200); ok = ld_rec(base + 2 * si, &r); }
                 if (!ok) { atomicExch(a.wait_failed, 1); r.s = 0.0; r.ecode = 2 * E_EMPTY + 1; r.flags = 0; }
-                bs[i] = r.s; be[i] = (r.ecode - 1) >> 1; fl |= r.flags; el = max(el, be[i]);
+                bs[i] = r.s; be[i] = (r.ecode - 1) >> 1; bu[i] = (double)rec_ub(r); fl |= r.flags & 1; el = max(el, be[i]);
             }
         }
         const int Em = redux_max(el);
@@ -905,7 +913,10 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
         // the slices' sums around the row's exponent, added in slice order
         double v = 0.0;
 #pragma unroll
-        for (int i = 0; i < SPL; ++i) { bs[i] = be[i] > E_EMPTY ? bs[i] * pow2d(max(be[i] - Em, -1000)) : 0.0; v += bs[i]; }
+        for (int i = 0; i < SPL; ++i) {
+            const double f = be[i] > E_EMPTY ? pow2d(max(be[i] - Em, -500)) : 0.0;
+            bs[i] *= f; bu[i] *= f * f; v += bs[i];
+        }
         double incl = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const double t2 = shfl_up_d(incl, o); if (lane >= o) incl += t2; }
@@ -953,9 +964,29 @@ __device__ __noinline__ void f_finish_seq(const FuseArgs& a, FShared& S, int b, 
     const FRow rp = pair ? shfl_row(sp, nn) : rb;
     FRow rq = shfl_row(sq, pair ? nn : 0);
     if (!pair) { rq.inv_s = 0.0; rq.e = E_EMPTY; rq.st = 0; }
-    // The draw's error bound wants sum p^2 + q^2 over the row pair.  A row's exponent is the integer nearest to its
-    // largest argument, so its largest probability is at most sqrt(2) / S, and sum p^2 <= max p * sum p = max p.
-    const double bound = draw_bound(1.4142135623730951 * (rp.inv_s + rq.inv_s), (double)a.kappa);
+    // The draw's error bound wants sum p^2 + q^2 over the row pair, for which the records carry an upper bound per slice
+    // (a chunk's e are at most sqrt(2) around its own exponent, so its sum of e^2 is at most sqrt(2) times its sum of e:
+    // chunks far below the row's largest logit count next to nothing, and a peaked row gets a bound close to the sum).
+    double s2 = 0.0;
+    if (pair) {
+        const FRec* base = a.rec + ((int64_t)du * T) * 2;
+#pragma unroll
+        for (int i = 0; i < SPL; ++i) {
+            const int si = lane * per + i;
+            if (i < per && si < T) {
+                FRec r0, r1;
+                ld_rec(base + 2 * si, &r0); ld_rec(base + 2 * si + 1, &r1);
+                const int e0 = (r0.ecode - 1) >> 1, e1 = (r1.ecode - 1) >> 1;
+                if (e0 > E_EMPTY && rp.e > E_EMPTY) { const double f = pow2d(max(e0 - rp.e, -500)) * rp.inv_s; s2 += (double)rec_ub(r0) * f * f; }
+                if (e1 > E_EMPTY && rq.e > E_EMPTY) { const double f = pow2d(max(e1 - rq.e, -500)) * rq.inv_s; s2 += (double)rec_ub(r1) * f * f; }
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < SPL; ++i) s2 += bu[i] * rp.inv_s * rp.inv_s;
+    }
+    s2 = warp_sum(s2);
+    const double bound = draw_bound(1.4142135623730951 * s2, (double)a.kappa);
     // the slices' masses (bonus row: sums of e around the row's exponent -> probabilities); the slice that owns u Z
     double sm[SPL];
 #pragma unroll
