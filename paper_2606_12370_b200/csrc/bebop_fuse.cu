@@ -1163,17 +1163,19 @@ bool fuse_supported(const RowArgs& a) {
 // Measured on a B200 against the pipelined kernel (about 0.4 GB of logits per call unless said otherwise):
 // bebop_tv is faster through the fused kernel at every shape tried with at most 32 slices per row (3 to 12 per cent
 // from 32,768 to 262,144 bf16 logits per row, twice as fast at 8,192 and below; fp32 alike), and slower with more
-// (the merge of a unit's records then takes several records per lane).  bebop_verify is faster up to about ten slices per row
-// (7 per cent at 65,536 bf16 logits, 15 at 32,768, twice as fast at 16,384 and below) and 3 to 8 per cent slower
-// from 100,000 on, where the pipelined kernel streams at close to the copy rate; small calls (a few dozen tasks per
-// CTA) are faster fused at any row length, tiny ones (fewer than two tasks per SM) through the pipelined kernel.
+// (the merge of a unit's records then takes several records per lane).  bebop_verify is faster up to eleven slices
+// per row (5 per cent at 90,112 bf16 logits, 7 at 65,536, 15 at 32,768, twice as fast at 16,384 and below) and 2
+// to 6 per cent slower from 100,000 on, where the pipelined kernel streams at close to the copy rate -- except with
+// one draft position per sequence, where half of the rows are bonus rows (5 to 13 per cent faster at 100,000 to
+// 262,144); small calls (a few dozen tasks per CTA) are faster fused at any row length, tiny ones (fewer than two
+// tasks per SM) through the pipelined kernel.
 bool fuse_preferred(const RowArgs& a, bool tv_only) {
     const int T = make_fuse_plan(a.B, a.K, a.nvec, 1).T;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return false; }
     const long long tasks = (long long)a.B * (tv_only ? 1 : a.K + 1) * T;
     if (T > 32 || tasks < 2LL * sms) return false;       // (a call of a few tasks is all start-up: 0.038 against 0.031 ms)
-    if (tv_only || T <= 10) return true;
+    if (tv_only || T <= 11 || a.K == 1) return true;
     return tasks <= 40LL * sms;
 }
 
